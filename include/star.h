@@ -1,0 +1,182 @@
+/*
+ * star.h — C ABI of the B200 grouped gradient aggregation + parameter update.
+ *
+ * The operation (STAR's parameter-server hot path).  A round hands the server W
+ * workers' gradient buffers and a SCHEDULE: an ordered list of disjoint,
+ * non-empty groups of workers.  SSGD is one group of all workers, ASGD is one
+ * group per worker in arrival order (paper Section I); the static x-order mode
+ * uses x workers per update and the dynamic x-order mode one worker cluster per
+ * update (Section I contribution (2), Section IV-B), clusters taken in
+ * ascending order of their slowest member (Section IV-C1, text before Eq. 2).
+ * For every element i and every group k in schedule order the library applies
+ *
+ *     s    = g[m_k0][i] + g[m_k1][i] + ...          members in listed order
+ *     gbar = s / |G_k|
+ *     d    = fma(wd, p[i], gbar)
+ *     v[i] = fma(mu, v[i], d)
+ *     p[i] = fma(-lr_k, v[i], p[i])
+ *
+ * each line one correctly rounded IEEE-754 binary32 operation (bf16 gradients
+ * are widened exactly first).  All groups of a round are fused into ONE pass:
+ * every scheduled gradient element and p, v are read once, p and v are written
+ * once: n * (sum_k |G_k| * sizeof(g) + 16) bytes of traffic per round.
+ *
+ * A schedule is a CSR pair: group k = group_members[group_offsets[k] ..
+ * group_offsets[k+1]).  It need not cover every worker (a round may use only
+ * the workers that reported); a worker may appear at most once.
+ *
+ * Conventions that hold for every entry point
+ *   - "device" pointers are CUDA device memory of the current device; "host"
+ *     arrays are ordinary memory that is read completely before the call
+ *     returns (the caller may free or reuse it at once).
+ *   - The caller owns every buffer.  The library allocates no device memory and
+ *     keeps no pointer after a call returns, except inside a caller-provided
+ *     workspace.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t; NULL = legacy default
+ *     stream) and the call returns without synchronizing.
+ *   - Every argument error is found on the host BEFORE anything is launched and
+ *     leaves p and v untouched.  STAR_ERR_CUDA is a failed launch or runtime
+ *     call; star_last_cuda_error() gives its cudaError_t.
+ *   - There is no CPU path: without a usable CUDA device the compute entry
+ *     points return STAR_ERR_CUDA.
+ *   - params, momentum and the scheduled gradient buffers must not overlap.
+ *     Element-size alignment is required (4 bytes fp32, 2 bytes bf16); 16-byte
+ *     aligned buffers take the vector path, others a slower scalar path with
+ *     identical results.
+ */
+#ifndef STAR_H_
+#define STAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    STAR_OK = 0,
+    STAR_ERR_NULL_POINTER = 1,      /* a required pointer is NULL */
+    STAR_ERR_INVALID_ARG = 2,       /* negative size, bad dtype, misaligned or overlapping buffers */
+    STAR_ERR_BAD_SCHEDULE = 3,      /* empty group, duplicate or out-of-range member, bad offsets */
+    STAR_ERR_UNSUPPORTED = 4,       /* W above STAR_MAX_WORKERS */
+    STAR_ERR_WORKSPACE_TOO_SMALL = 5,
+    STAR_ERR_CUDA = 6               /* see star_last_cuda_error() */
+} star_status_t;
+
+typedef enum { STAR_DTYPE_F32 = 0, STAR_DTYPE_BF16 = 1 } star_dtype_t;
+
+#define STAR_MAX_WORKERS 64
+
+/* Static, NUL-terminated name of a status code. */
+const char *star_status_string(star_status_t status);
+
+/* cudaError_t of the most recent STAR_ERR_CUDA on the calling thread (0 if none). */
+int star_last_cuda_error(void);
+
+/* Number of kernels this library has launched in the calling process so far. */
+int64_t star_launch_count(void);
+
+/* ---------------------------------------------------------------------------
+ * Schedule encoding (host only; no CUDA call).  Turns a synchronization-mode
+ * decision into the CSR pair.  offsets_out needs room for W + 1 entries,
+ * members_out for W entries; *n_groups_out receives K.
+ * ------------------------------------------------------------------------- */
+
+/* STAR_OK iff the pair describes n_groups non-empty, pairwise disjoint groups
+ * of workers in [0, W) with group_offsets[0] == 0 (Section IV-B: a gradient
+ * report feeds exactly one update).  n_groups == 0 is valid. */
+star_status_t star_schedule_validate(const int32_t *group_offsets, const int32_t *group_members,
+                                     int n_groups, int W);
+
+/* Static x-order mode (Section IV-B): consecutive runs of x workers of
+ * arrival_order (n_arrived distinct workers, earliest first; NULL = 0..W-1 with
+ * n_arrived = W).  x == n_arrived gives SSGD, x == 1 ASGD (Section I).  If x
+ * does not divide n_arrived the last group is smaller.  sort_members != 0 lists
+ * each group's members in ascending worker index, otherwise in arrival order. */
+star_status_t star_schedule_static_x(const int32_t *arrival_order, int n_arrived, int W, int x,
+                                     int sort_members, int32_t *offsets_out,
+                                     int32_t *members_out, int *n_groups_out);
+
+/* Groups from a per-worker label group_of_worker[W] (-1 = worker absent):
+ * groups in ascending label order, members in ascending worker index. */
+star_status_t star_schedule_from_labels(const int32_t *group_of_worker, int W,
+                                        int32_t *offsets_out, int32_t *members_out,
+                                        int *n_groups_out);
+
+/* Dynamic x-order mode (Section IV-B, ordering of Section IV-C1): one group per
+ * cluster id in cluster_of_worker[W] (-1 = absent), groups ascending in the
+ * cluster's largest iter_time; ties go to the cluster holding the smaller
+ * worker index; members in ascending worker index.  iter_time must be finite. */
+star_status_t star_schedule_dynamic_x(const double *iter_time, const int32_t *cluster_of_worker,
+                                      int W, int32_t *offsets_out, int32_t *members_out,
+                                      int *n_groups_out);
+
+/* ---------------------------------------------------------------------------
+ * Fused grouped update of one flat tensor (the operation defined at the top).
+ *   params, momentum : device, fp32, n elements, updated in place
+ *   grads            : host array of W device pointers, n elements of
+ *                      grad_dtype each; entries of unscheduled workers are
+ *                      never dereferenced and may be NULL
+ *   group_offsets    : host, n_groups + 1 entries;  group_members : host
+ *   lr, mu, wd       : learning rate, momentum coefficient, weight decay
+ * n == 0 or n_groups == 0 is a successful no-op.  One kernel launch.
+ * ------------------------------------------------------------------------- */
+star_status_t star_group_update(float *params, float *momentum, const void *const *grads, int W,
+                                star_dtype_t grad_dtype, int64_t n,
+                                const int32_t *group_offsets, const int32_t *group_members,
+                                int n_groups, float lr, float mu, float wd, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Fused grouped update of a LIST of tensors (per-layer parameters) in one
+ * launch.  The pointer table and tile map live in a caller-provided device
+ * workspace that is prepared once per tensor list and reused every round.
+ * ------------------------------------------------------------------------- */
+
+/* Host-side description of a prepared tensor list.  Plain data, filled by
+ * star_multi_prepare and passed back by value-pointer every round; it holds
+ * the workspace address but owns nothing. */
+typedef struct {
+    uint64_t magic;            /* set by star_multi_prepare; anything else is rejected */
+    const void *d_workspace;   /* the caller's device workspace */
+    int64_t total_elements;    /* sum of the tensor sizes */
+    int64_t n_tiles;           /* work items the kernel walks */
+    int32_t n_tensors;
+    int32_t W;
+    int32_t grad_dtype;        /* star_dtype_t */
+    int32_t tile_elements;     /* elements per tile */
+} star_multi_plan_t;
+
+/* Bytes of device workspace needed for n_tensors tensors of the given sizes
+ * (host array, elements per tensor, 0 allowed) and W workers. */
+star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *sizes, int W,
+                                         size_t *bytes_out);
+
+/* Fill the workspace and *plan_out.  params, momentum: host arrays of n_tensors
+ * device pointers; grads: host array of n_tensors * W device pointers, entry
+ * [t * W + w] = worker w's gradient for tensor t (NULL allowed for workers that
+ * will never be scheduled); sizes: host, elements per tensor.  d_workspace:
+ * device, 256-byte aligned, at least star_multi_workspace_bytes() bytes.  The
+ * table is built in ordinary host memory and copied with one cudaMemcpyAsync on
+ * cuda_stream; the host copy is released before the call returns (a copy from
+ * pageable memory returns once the data is staged), later work on the same
+ * stream sees the table.  Not a per-round call: once per tensor list. */
+star_status_t star_multi_prepare(int n_tensors, float *const *params, float *const *momentum,
+                                 const void *const *grads, const int64_t *sizes, int W,
+                                 star_dtype_t grad_dtype, void *d_workspace,
+                                 size_t workspace_bytes, void *cuda_stream,
+                                 star_multi_plan_t *plan_out);
+
+/* One round over the prepared list: the same operation as star_group_update on
+ * every tensor, one kernel launch in total.  A scheduled worker whose gradient
+ * pointer was NULL at prepare time is rejected with STAR_ERR_NULL_POINTER only
+ * if it was NULL for every tensor; mixed cases are the caller's error. */
+star_status_t star_group_update_multi(const star_multi_plan_t *plan,
+                                      const int32_t *group_offsets, const int32_t *group_members,
+                                      int n_groups, float lr, float mu, float wd,
+                                      void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STAR_H_ */

@@ -1,0 +1,167 @@
+/*
+ * CPU oracle for STAR's parameter-server-side grouped aggregation + update.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, serial, obviously-correct
+ * statement of what the grouped update computes.  It is compiled with gcc,
+ * called from the test-suite, the smoke check and the CPU-baseline leg of the
+ * benchmark, and from nowhere else.  It shares no code, header, table or
+ * helper with the CUDA library and neither side includes the other.
+ *
+ * What it follows (paper: "Straggler Tolerant and Resilient DL Training on
+ * Homogeneous GPUs"):
+ *   - Section I:    SSGD updates parameters only once gradients from all N
+ *                   workers are in; ASGD updates on the gradient of any one
+ *                   worker.
+ *   - Section I, contribution (2) and Section IV-B: the static x-order mode
+ *                   uses the gradients of x workers for each parameter update;
+ *                   the dynamic x-order mode uses the gradient reports of one
+ *                   worker cluster for each update.
+ *   - Section IV-C1 (text before Eq. 2): clusters are taken in ascending
+ *                   order of their largest iteration time, i.e. the groups of
+ *                   a round are ORDERED and are applied one after another.
+ *   - Section II:   the PS updates the parameters (one master copy).
+ *
+ * The paper never prints the update rule.  The reading used here: every group
+ * update is one complete SGD step with momentum (dampening 0, no Nesterov)
+ * and L2 weight decay folded into the gradient, on the MEAN of the group's
+ * gradients:
+ *
+ *     for k = 0 .. K-1 (schedule order):
+ *         s    = g[m_k0][i] + g[m_k1][i] + ...      (left to right, CSR order)
+ *         gbar = s / |G_k|
+ *         d    = gbar + wd * p[i]
+ *         v[i] = mu * v[i] + d
+ *         p[i] = p[i] - lr * v[i]
+ *
+ * Two variants:
+ *   oracle_group_update_f32  canonical binary32 sequence; each line above is
+ *                            ONE correctly rounded IEEE operation: fp32 add,
+ *                            fp32 true division, and three fused multiply-adds
+ *                            d=fma(wd,p,gbar), v=fma(mu,v,d), p=fma(-lr,v,p).
+ *   oracle_group_update_f64  the same loop in binary64 without fused
+ *                            operations: the shadow that says how far the
+ *                            fp32 sequence is from the real-number result.
+ *
+ * Pins (tests/test_oracle_pins.py): hand-worked dyadic example, exact-rational
+ * brute force, closed forms (mu=wd=0; wd=0; 2x2 affine recurrence), the
+ * library SGD optimizer of PyTorch in fp64, SSGD == one mean update, fused K
+ * groups == K single-group calls, member-permutation invariance.
+ *
+ * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+enum { ORACLE_DTYPE_F32 = 0, ORACLE_DTYPE_BF16 = 1 };
+
+/* bf16 is the upper half of a binary32: widening is exact. */
+static float widen_bf16(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+static float grad_at(const void *buf, int dtype, int64_t i)
+{
+    if (dtype == ORACLE_DTYPE_BF16)
+        return widen_bf16(((const uint16_t *)buf)[i]);
+    return ((const float *)buf)[i];
+}
+
+/* 1 if the schedule is one the definition covers, else 0.  The public
+ * functions return 0 on success and 1 on such a schedule. */
+static int schedule_ok(const int32_t *group_offsets, const int32_t *group_members,
+                       int n_groups, int W)
+{
+    if (n_groups < 0 || W < 0)
+        return 0;
+    if (n_groups == 0)
+        return 1;
+    if (!group_offsets || !group_members || group_offsets[0] != 0)
+        return 0;
+    for (int k = 0; k < n_groups; ++k)
+        if (group_offsets[k + 1] <= group_offsets[k])
+            return 0; /* the mean of an empty group is undefined */
+    for (int j = 0; j < group_offsets[n_groups]; ++j) {
+        if (group_members[j] < 0 || group_members[j] >= W)
+            return 0;
+        for (int l = 0; l < j; ++l)
+            if (group_members[l] == group_members[j])
+                return 0; /* a gradient report feeds exactly one update */
+    }
+    return 1;
+}
+
+/*
+ * Canonical binary32 oracle.  lrs has one learning rate per group (Section
+ * IV-C1, "Scaling learning rate after switching": the rate follows the number
+ * of gradient reports y used by the update); pass the same value K times for
+ * a single rate.  snapshots is NULL, or K pointers of which the non-NULL ones
+ * receive the parameters as they stand right after that group's update: the
+ * copy the PS sends back to the workers of that group (Section II).
+ */
+int oracle_group_update_f32(float *params, float *momentum,
+                            const void *const *grads, int W, int grad_dtype,
+                            int64_t n, const int32_t *group_offsets,
+                            const int32_t *group_members, int n_groups,
+                            const float *lrs, float mu, float wd,
+                            float *const *snapshots)
+{
+    if (!schedule_ok(group_offsets, group_members, n_groups, W))
+        return 1;
+    for (int64_t i = 0; i < n; ++i) {
+        float p = params[i];
+        float v = momentum[i];
+        for (int k = 0; k < n_groups; ++k) {
+            const int first = group_offsets[k];
+            const int last = group_offsets[k + 1];
+            float s = grad_at(grads[group_members[first]], grad_dtype, i);
+            for (int j = first + 1; j < last; ++j)
+                s = s + grad_at(grads[group_members[j]], grad_dtype, i);
+            const float gbar = s / (float)(last - first);
+            const float d = fmaf(wd, p, gbar);
+            v = fmaf(mu, v, d);
+            p = fmaf(-lrs[k], v, p);
+            if (snapshots && snapshots[k])
+                snapshots[k][i] = p;
+        }
+        params[i] = p;
+        momentum[i] = v;
+    }
+    return 0;
+}
+
+/* Binary64 shadow: same order, plain multiply and add, no fused operation. */
+int oracle_group_update_f64(double *params, double *momentum,
+                            const void *const *grads, int W, int grad_dtype,
+                            int64_t n, const int32_t *group_offsets,
+                            const int32_t *group_members, int n_groups,
+                            const double *lrs, double mu, double wd,
+                            double *const *snapshots)
+{
+    if (!schedule_ok(group_offsets, group_members, n_groups, W))
+        return 1;
+    for (int64_t i = 0; i < n; ++i) {
+        double p = params[i];
+        double v = momentum[i];
+        for (int k = 0; k < n_groups; ++k) {
+            const int first = group_offsets[k];
+            const int last = group_offsets[k + 1];
+            double s = (double)grad_at(grads[group_members[first]], grad_dtype, i);
+            for (int j = first + 1; j < last; ++j)
+                s = s + (double)grad_at(grads[group_members[j]], grad_dtype, i);
+            const double gbar = s / (double)(last - first);
+            const double d = gbar + wd * p;
+            v = mu * v + d;
+            p = p - lrs[k] * v;
+            if (snapshots && snapshots[k])
+                snapshots[k][i] = p;
+        }
+        params[i] = p;
+        momentum[i] = v;
+    }
+    return 0;
+}

@@ -1,0 +1,137 @@
+"""numpy front end of the C oracle in ``star_oracle.c``.
+
+TEST INFRASTRUCTURE ONLY (see the header of ``star_oracle.c``).  This module
+compiles the C file with gcc on first use and marshals numpy arrays into it.
+It holds no arithmetic of its own.
+
+bf16 gradients travel as ``numpy.uint16`` arrays holding the raw bit patterns;
+fp32 gradients as ``numpy.float32`` arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "star_oracle.c")
+_LIB = os.path.join(_HERE, "libstar_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+DTYPE_F32 = 0
+DTYPE_BF16 = 1
+
+# IEEE sequence must survive the compiler: no contraction, no fast-math.
+CFLAGS = ["-O2", "-ffp-contract=off", "-fno-fast-math", "-Wall", "-Wextra",
+          "-shared", "-fPIC"]
+
+
+def build(force: bool = False) -> str:
+    """Compile ``star_oracle.c`` into ``libstar_oracle.so`` beside it."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)
+                 or os.path.getmtime(_LIB) < os.path.getmtime(_SRC))
+        if force or stale:
+            tmp = _LIB + ".tmp.%d" % os.getpid()
+            subprocess.check_call(["gcc", *CFLAGS, "-o", tmp, _SRC, "-lm"])
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        common = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                  ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
+                  ctypes.c_int, ctypes.c_void_p]
+        lib.oracle_group_update_f32.argtypes = common + [
+            ctypes.c_float, ctypes.c_float, ctypes.c_void_p]
+        lib.oracle_group_update_f32.restype = ctypes.c_int
+        lib.oracle_group_update_f64.argtypes = common + [
+            ctypes.c_double, ctypes.c_double, ctypes.c_void_p]
+        lib.oracle_group_update_f64.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _grad_dtype(grads: Sequence[Optional[np.ndarray]]) -> int:
+    kinds = {g.dtype for g in grads if g is not None}
+    if kinds == {np.dtype(np.float32)}:
+        return DTYPE_F32
+    if kinds == {np.dtype(np.uint16)}:
+        return DTYPE_BF16
+    raise TypeError("gradients must all be float32, or all uint16 (bf16 bits): %r" % kinds)
+
+
+def _call(fn, real, params, momentum, grads, group_offsets, group_members, lrs, mu, wd,
+          snapshots):
+    n = params.shape[0]
+    if params.dtype != real or momentum.dtype != real:
+        raise TypeError("params/momentum must be %s" % real)
+    if momentum.shape != (n,) or params.ndim != 1:
+        raise ValueError("params and momentum must be 1-D of equal length")
+    for a in (params, momentum):
+        if not a.flags.c_contiguous or not a.flags.writeable:
+            raise ValueError("params/momentum must be contiguous and writeable")
+    W = len(grads)
+    dt = _grad_dtype(grads)
+    ptrs = (ctypes.c_void_p * max(W, 1))()
+    keep = []
+    for w, g in enumerate(grads):
+        if g is None:
+            ptrs[w] = None
+            continue
+        if g.shape != (n,) or not g.flags.c_contiguous:
+            raise ValueError("gradient %d must be contiguous with %d elements" % (w, n))
+        keep.append(g)
+        ptrs[w] = g.ctypes.data
+    off = np.ascontiguousarray(group_offsets, dtype=np.int32)
+    mem = np.ascontiguousarray(group_members, dtype=np.int32)
+    K = off.shape[0] - 1 if off.shape[0] > 0 else 0
+    lr_arr = np.ascontiguousarray(np.broadcast_to(np.asarray(lrs, dtype=real), (max(K, 0),)))
+    for w in mem[: off[K] if K > 0 else 0]:
+        if 0 <= w < W and grads[w] is None:
+            raise ValueError("scheduled worker %d has no gradient buffer" % w)
+    snap_ptrs = None
+    if snapshots is not None:
+        if len(snapshots) != K:
+            raise ValueError("snapshots needs one entry (array or None) per group")
+        snap_ptrs = (ctypes.c_void_p * max(K, 1))()
+        for k, s in enumerate(snapshots):
+            if s is None:
+                snap_ptrs[k] = None
+                continue
+            if s.dtype != real or s.shape != (n,) or not s.flags.c_contiguous:
+                raise ValueError("snapshot %d has the wrong dtype or shape" % k)
+            snap_ptrs[k] = s.ctypes.data
+    rc = fn(params.ctypes.data, momentum.ctypes.data, ptrs, W, dt, n,
+            off.ctypes.data, mem.ctypes.data, K, lr_arr.ctypes.data,
+            mu, wd, snap_ptrs)
+    if rc != 0:
+        raise ValueError("schedule outside the definition (empty group, duplicate or "
+                         "out-of-range member)")
+
+
+def group_update_f32(params, momentum, grads, group_offsets, group_members, lrs, mu, wd,
+                     snapshots=None):
+    """Canonical binary32 grouped update, in place on ``params`` / ``momentum``.
+
+    ``lrs`` is a scalar or one learning rate per group.  ``mu`` and ``wd`` are
+    rounded to binary32 on the way in, as the C signature takes floats.
+    """
+    _call(_load().oracle_group_update_f32, np.float32, params, momentum, grads,
+          group_offsets, group_members, lrs, float(np.float32(mu)), float(np.float32(wd)),
+          snapshots)
+
+
+def group_update_f64(params, momentum, grads, group_offsets, group_members, lrs, mu, wd,
+                     snapshots=None):
+    """Binary64 shadow of the same loop, in place on float64 arrays."""
+    _call(_load().oracle_group_update_f64, np.float64, params, momentum, grads,
+          group_offsets, group_members, lrs, float(mu), float(wd), snapshots)
