@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the fused grouped aggregate + update.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
+                    [--impl ours|reference] [--no-extra]
+
+A step is one round of the whole path on one batch of synthetic gradients:
+the mode decision of the round is encoded into a CSR schedule (host, in the
+library) and the fused update kernel is launched once.  Prints ONE JSON line.
+
+  value      achieved GB/s = algorithmic bytes / device time, inputs resident
+             in HBM; bytes per round = n * (sum_k |G_k| * sizeof(g) + 16)
+  e2e        the same metric through the host-buffer entry point: parameters,
+             momentum and gradients start in pinned host memory, results end
+             there, every copy inside the timed region
+  roofline   the update kernel against the measured HBM copy bandwidth
+  cpu_baseline  the CPU oracle timed on this machine's cores (reported only)
+
+With N > 1 (under torchrun) every rank runs the same workload on its own GPU
+(the path is elementwise: shards need no exchange), the time is the maximum
+over ranks and the value the sum of all ranks' bytes over that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "grouped aggregate+update HBM GB/s"
+UNIT = "GB/s"
+HEADLINE = "cfg1_resnet50"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------
+# clocks during the timed region
+# ---------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the
+    timed region runs."""
+
+    REASONS = (("sw_power_cap", 0x4), ("hw_slowdown", 0x8), ("sw_thermal_slowdown", 0x20),
+               ("hw_thermal_slowdown", 0x40), ("hw_power_brake", 0x80))
+
+    def __init__(self, index: int, period: float = 0.01):
+        self.index, self.period = index, period
+        self.sm, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible:
+                ids = [x for x in visible.split(",") if x.strip()]
+                if index < len(ids) and ids[index].strip().isdigit():
+                    phys = int(ids[index])
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                for name, bit in self.REASONS:
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.sm), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+# ---------------------------------------------------------------------------
+# device side
+# ---------------------------------------------------------------------------
+class DeviceWorkload:
+    """One workload resident on the current device, ready to step."""
+
+    def __init__(self, w, grad_sets: int):
+        import torch
+        from paper_2512_09685_b200 import binding as B
+        from paper_2512_09685_b200 import workloads as WL
+        self.torch, self.B, self.w = torch, B, w
+        dev = "cuda"
+        self.params = WL.make_params(w, dev)
+        self.momentum = WL.make_momentum(w, dev)
+        dt = w.torch_grad_dtype()
+        self.grad_sets = []
+        for s in range(grad_sets):
+            one = []
+            for wk in range(w.W):
+                bufs = [torch.empty(size, dtype=dt, device=dev) for size in w.sizes]
+                WL.fill_grads(w, s, wk, bufs)
+                one.append(bufs)
+            self.grad_sets.append(one)
+        self.plans = None
+        if w.multi_tensor:
+            self.workspaces, self.plans = [], []
+            for one in self.grad_sets:
+                ws = torch.empty(B.star_multi_workspace_bytes(w.sizes, w.W), dtype=torch.uint8, device=dev)
+                self.workspaces.append(ws)
+                self.plans.append(B.star_multi_prepare(self.params, self.momentum, one, ws))
+        else:
+            self.flat_grads = [[bufs[0] for bufs in one] for one in self.grad_sets]
+        self.step_index = 0
+        torch.cuda.synchronize()
+
+    def step(self) -> int:
+        """One round: encode the decision, launch the fused update.  Returns the
+        number of scheduled workers (for the byte count)."""
+        w, B = self.w, self.B
+        off, mem = B.encode(w.decision(self.step_index))
+        which = self.step_index % len(self.grad_sets)
+        if self.plans is not None:
+            B.star_group_update_multi(self.plans[which], off, mem, w.lr, w.mu, w.wd)
+        else:
+            B.star_group_update(self.params[0], self.momentum[0], self.flat_grads[which], off, mem,
+                                w.lr, w.mu, w.wd)
+        self.step_index += 1
+        return off[-1]
+
+    def reset_state(self):
+        # keeps values bounded over thousands of timed rounds; not timed
+        for v in self.momentum:
+            v.zero_()
+
+
+def time_device(dw: DeviceWorkload, steps: int, warmup: int, dist, sampler=None):
+    """Returns (seconds for `steps` rounds [max over ranks], per-launch ms list,
+    algorithmic bytes of those rounds on this rank, launches)."""
+    torch, B = dw.torch, dw.B
+    for _ in range(warmup):
+        dw.step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    launches0 = B.star_launch_count()
+    scheduled = 0
+    if sampler is not None:
+        sampler.__enter__()
+    events[0].record()
+    for i in range(steps):
+        scheduled += dw.step()
+        events[i + 1].record()
+    torch.cuda.synchronize()
+    if sampler is not None:
+        sampler.__exit__(None, None, None)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches = B.star_launch_count() - launches0
+    total_ms = events[0].elapsed_time(events[steps])
+    per_launch = [events[i].elapsed_time(events[i + 1]) for i in range(steps)]
+    nbytes = dw.w.n * (scheduled * dw.w.grad_bytes + 16 * steps)
+    seconds = total_ms / 1e3
+    if dist is not None:
+        t = torch.tensor([seconds], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        seconds = float(t.item())
+    return seconds, per_launch, nbytes, launches
+
+
+# ---------------------------------------------------------------------------
+# CPU oracle timing
+# ---------------------------------------------------------------------------
+def time_oracle(w, n_sample: int, min_seconds: float, threads: int):
+    """The oracle, as it stands, on the first `n_sample` elements of workload
+    `w` (inputs generated on the CPU), `threads` Python threads over disjoint
+    index ranges (the C call releases the GIL).  Returns (GB/s, elements/s,
+    rounds run, seconds)."""
+    import numpy as np
+    import torch
+    from oracle import schedule as S
+    from oracle import star_oracle as O
+    from paper_2512_09685_b200 import workloads as WL
+
+    ws = WL.scaled(w, n_sample)
+    p = WL.make_params(ws, "cpu")[0].numpy()
+    v = WL.make_momentum(ws, "cpu")[0].numpy()
+    grads = []
+    for g in WL.make_grads(ws, 0, "cpu"):
+        g = g[0]
+        grads.append(g.view(torch.int16).numpy().view(np.uint16) if g.dtype == torch.bfloat16 else g.numpy())
+    bounds = [n_sample * i // threads for i in range(threads + 1)]
+
+    def encode(step):
+        d = w.decision(step)
+        if d.kind == "labels":
+            return S.from_labels(d.labels)
+        return S.static_x(d.arrival_order, d.W, d.x, d.sort_members)
+
+    def one_round(step):
+        off, mem = encode(step)
+        lr = np.float32(w.lr)
+        def work(i):
+            a, b = bounds[i], bounds[i + 1]
+            O.group_update_f32(p[a:b], v[a:b], [g[a:b] for g in grads], off, mem, lr, w.mu, w.wd)
+        if threads == 1:
+            work(0)
+        else:
+            ts = [threading.Thread(target=work, args=(i,)) for i in range(threads)]
+            for t in ts:
+                t.start()
+            for t in ts:
+                t.join()
+        return off[-1]
+
+    one_round(0)                                   # warm-up (also builds the oracle)
+    rounds, scheduled = 0, 0
+    t0 = time.perf_counter()
+    while True:
+        scheduled += one_round(rounds + 1)
+        rounds += 1
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds:
+            break
+    nbytes = n_sample * (scheduled * w.grad_bytes + 16 * rounds)
+    return nbytes / dt / 1e9, n_sample * rounds / dt, rounds, dt
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+# ---------------------------------------------------------------------------
+def run_reference(args, rank: int):
+    """--impl reference: the CPU oracle on the host cores."""
+    if rank != 0:
+        return
+    from paper_2512_09685_b200 import workloads as WL
+    w = WL.BY_NAME[args.workload]
+    cores = host_cores()
+    n_sample = min(w.n, 4_000_000)
+    per_step = []
+    for _ in range(max(args.warmup, 0)):
+        time_oracle(w, n_sample, 0.0, cores)
+    t0 = time.perf_counter()
+    gbs_acc = []
+    for _ in range(args.steps):
+        gbs, eps, rounds, dt = time_oracle(w, n_sample, 0.0, cores)
+        gbs_acc.append(gbs)
+        per_step.append(dt / rounds * 1e3)
+    value = statistics.mean(gbs_acc)
+    sample = "first %d of %d elements of %s per step, %d threads over disjoint ranges" % (
+        n_sample, w.n, w.name, cores)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(per_step),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": w.name, "model": w.model, "n": w.n, "W": w.W,
+                                        "grad_dtype": w.grad_dtype, "sample_elements": n_sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default=HEADLINE)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the other workloads, the CPU baseline and the end-to-end leg")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    from paper_2512_09685_b200 import binding as B        # raises if the CUDA library is missing
+    from paper_2512_09685_b200 import workloads as WL
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    if max(args.warmup, 0) < 3:
+        args.warmup = 3
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist = dist_mod
+
+    w = WL.BY_NAME[args.workload]
+    peak, peak_kind = measured_peak()
+    dw = DeviceWorkload(w, grad_sets=2 if w.n * w.W * w.grad_bytes < (4 << 30) else 1)
+    sampler = ClockSampler(local_rank)
+    seconds, per_launch, nbytes, launches = time_device(dw, args.steps, args.warmup, dist, sampler)
+    gbs_rank = nbytes / seconds / 1e9
+    value = gbs_rank * world
+    kernel_ms = statistics.mean(per_launch)
+    achieved = (nbytes / args.steps) / (kernel_ms / 1e3) / 1e9
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "model": w.model, "n": w.n, "W": w.W, "grad_dtype": w.grad_dtype,
+                   "tensors": len(w.sizes), "bytes_per_step": nbytes // args.steps,
+                   "l2": "inputs larger than L2: %.0f MB per step, gradient buffer sets rotated: %d" % (
+                       nbytes / args.steps / 1e6, len(dw.grad_sets)),
+                   "parallelism": "replicas x%d" % world},
+        "param_elements_per_s": w.n * args.steps * world / seconds,
+        "pct_of_peak": {"measured_%.1f" % peak: 100 * gbs_rank / peak, "datasheet_8000": 100 * gbs_rank / 8000},
+        "gpu_launches": launches,
+        "clocks": sampler.summary(),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_kind": "of " + peak_kind,
+                     "kernel": "star_update_multi_kernel" if w.multi_tensor else "star_update_flat_kernel",
+                     "kernel_ms_mean": kernel_ms, "kernel_ms_median": statistics.median(per_launch),
+                     "kernel_ms_min": min(per_launch)},
+    }
+
+    if not args.no_extra and rank == 0 and world == 1:
+        del dw
+        torch.cuda.empty_cache()
+        others = {}
+        for other in WL.WORKLOADS:
+            if other.name == w.name:
+                continue
+            odw = DeviceWorkload(other, grad_sets=1 if other.n > 30_000_000 else 8)
+            osteps = 50 if other.n > 30_000_000 else 400
+            osec, oper, obytes, _ = time_device(odw, osteps, 5, None)
+            ogbs = obytes / osec / 1e9
+            others[other.name] = {"gbs": ogbs, "frac_of_%s_peak" % peak_kind: ogbs / peak,
+                                  "ms_per_step": osec / osteps * 1e3,
+                                  "param_elements_per_s": other.n * osteps / osec, "steps": osteps}
+            del odw
+            torch.cuda.empty_cache()
+        out["other_workloads"] = others
+        cores = host_cores()
+        n_sample = min(w.n, 8_000_000)
+        cgbs, ceps, rounds, cdt = time_oracle(w, n_sample, 8.0, cores)
+        sgbs, seps, srounds, sdt = time_oracle(w, n_sample, 4.0, 1)
+        out["cpu_baseline"] = {
+            "value": cgbs, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "first %d of %d elements of %s, %d rounds in %.1f s, %d threads over disjoint ranges"
+                      % (n_sample, w.n, w.name, rounds, cdt, cores),
+            "param_elements_per_s": ceps,
+            "single_thread": {"value": sgbs, "param_elements_per_s": seps, "rounds": srounds}}
+
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -50,6 +50,12 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#if defined(__GNUC__)
+#define STAR_API __attribute__((visibility("default")))
+#else
+#define STAR_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -69,13 +75,13 @@ typedef enum { STAR_DTYPE_F32 = 0, STAR_DTYPE_BF16 = 1 } star_dtype_t;
 #define STAR_MAX_WORKERS 64
 
 /* Static, NUL-terminated name of a status code. */
-const char *star_status_string(star_status_t status);
+STAR_API const char *star_status_string(star_status_t status);
 
 /* cudaError_t of the most recent STAR_ERR_CUDA on the calling thread (0 if none). */
-int star_last_cuda_error(void);
+STAR_API int star_last_cuda_error(void);
 
 /* Number of kernels this library has launched in the calling process so far. */
-int64_t star_launch_count(void);
+STAR_API int64_t star_launch_count(void);
 
 /* ---------------------------------------------------------------------------
  * Schedule encoding (host only; no CUDA call).  Turns a synchronization-mode
@@ -86,7 +92,7 @@ int64_t star_launch_count(void);
 /* STAR_OK iff the pair describes n_groups non-empty, pairwise disjoint groups
  * of workers in [0, W) with group_offsets[0] == 0 (Section IV-B: a gradient
  * report feeds exactly one update).  n_groups == 0 is valid. */
-star_status_t star_schedule_validate(const int32_t *group_offsets, const int32_t *group_members,
+STAR_API star_status_t star_schedule_validate(const int32_t *group_offsets, const int32_t *group_members,
                                      int n_groups, int W);
 
 /* Static x-order mode (Section IV-B): consecutive runs of x workers of
@@ -94,13 +100,13 @@ star_status_t star_schedule_validate(const int32_t *group_offsets, const int32_t
  * n_arrived = W).  x == n_arrived gives SSGD, x == 1 ASGD (Section I).  If x
  * does not divide n_arrived the last group is smaller.  sort_members != 0 lists
  * each group's members in ascending worker index, otherwise in arrival order. */
-star_status_t star_schedule_static_x(const int32_t *arrival_order, int n_arrived, int W, int x,
+STAR_API star_status_t star_schedule_static_x(const int32_t *arrival_order, int n_arrived, int W, int x,
                                      int sort_members, int32_t *offsets_out,
                                      int32_t *members_out, int *n_groups_out);
 
 /* Groups from a per-worker label group_of_worker[W] (-1 = worker absent):
  * groups in ascending label order, members in ascending worker index. */
-star_status_t star_schedule_from_labels(const int32_t *group_of_worker, int W,
+STAR_API star_status_t star_schedule_from_labels(const int32_t *group_of_worker, int W,
                                         int32_t *offsets_out, int32_t *members_out,
                                         int *n_groups_out);
 
@@ -108,7 +114,7 @@ star_status_t star_schedule_from_labels(const int32_t *group_of_worker, int W,
  * cluster id in cluster_of_worker[W] (-1 = absent), groups ascending in the
  * cluster's largest iter_time; ties go to the cluster holding the smaller
  * worker index; members in ascending worker index.  iter_time must be finite. */
-star_status_t star_schedule_dynamic_x(const double *iter_time, const int32_t *cluster_of_worker,
+STAR_API star_status_t star_schedule_dynamic_x(const double *iter_time, const int32_t *cluster_of_worker,
                                       int W, int32_t *offsets_out, int32_t *members_out,
                                       int *n_groups_out);
 
@@ -122,7 +128,7 @@ star_status_t star_schedule_dynamic_x(const double *iter_time, const int32_t *cl
  *   lr, mu, wd       : learning rate, momentum coefficient, weight decay
  * n == 0 or n_groups == 0 is a successful no-op.  One kernel launch.
  * ------------------------------------------------------------------------- */
-star_status_t star_group_update(float *params, float *momentum, const void *const *grads, int W,
+STAR_API star_status_t star_group_update(float *params, float *momentum, const void *const *grads, int W,
                                 star_dtype_t grad_dtype, int64_t n,
                                 const int32_t *group_offsets, const int32_t *group_members,
                                 int n_groups, float lr, float mu, float wd, void *cuda_stream);
@@ -141,6 +147,7 @@ typedef struct {
     const void *d_workspace;   /* the caller's device workspace */
     int64_t total_elements;    /* sum of the tensor sizes */
     int64_t n_tiles;           /* work items the kernel walks */
+    uint64_t complete_workers; /* bit w set: worker w has a gradient for every non-empty tensor */
     int32_t n_tensors;
     int32_t W;
     int32_t grad_dtype;        /* star_dtype_t */
@@ -149,7 +156,7 @@ typedef struct {
 
 /* Bytes of device workspace needed for n_tensors tensors of the given sizes
  * (host array, elements per tensor, 0 allowed) and W workers. */
-star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *sizes, int W,
+STAR_API star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *sizes, int W,
                                          size_t *bytes_out);
 
 /* Fill the workspace and *plan_out.  params, momentum: host arrays of n_tensors
@@ -161,17 +168,18 @@ star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *sizes, in
  * cuda_stream; the host copy is released before the call returns (a copy from
  * pageable memory returns once the data is staged), later work on the same
  * stream sees the table.  Not a per-round call: once per tensor list. */
-star_status_t star_multi_prepare(int n_tensors, float *const *params, float *const *momentum,
+STAR_API star_status_t star_multi_prepare(int n_tensors, float *const *params, float *const *momentum,
                                  const void *const *grads, const int64_t *sizes, int W,
                                  star_dtype_t grad_dtype, void *d_workspace,
                                  size_t workspace_bytes, void *cuda_stream,
                                  star_multi_plan_t *plan_out);
 
 /* One round over the prepared list: the same operation as star_group_update on
- * every tensor, one kernel launch in total.  A scheduled worker whose gradient
- * pointer was NULL at prepare time is rejected with STAR_ERR_NULL_POINTER only
- * if it was NULL for every tensor; mixed cases are the caller's error. */
-star_status_t star_group_update_multi(const star_multi_plan_t *plan,
+ * every tensor, one kernel launch in total.  Scheduling a worker whose gradient
+ * pointer was NULL for some non-empty tensor at prepare time is rejected with
+ * STAR_ERR_NULL_POINTER.  A plan not made by star_multi_prepare is rejected
+ * with STAR_ERR_INVALID_ARG. */
+STAR_API star_status_t star_group_update_multi(const star_multi_plan_t *plan,
                                       const int32_t *group_offsets, const int32_t *group_members,
                                       int n_groups, float lr, float mu, float wd,
                                       void *cuda_stream);

@@ -1,0 +1,279 @@
+"""ctypes binding of ``libstar.so`` (declared in ``include/star.h``).
+
+Argument marshalling only: every function here has the name of the C entry
+point it forwards to, turns torch tensors into device pointers and Python lists
+into host arrays, and raises :class:`StarError` on a non-zero status.  PyTorch
+supplies device memory and the current stream; nothing is computed in Python
+and there is no fallback: if the library is missing, importing this module
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+from .workloads import ModeDecision
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libstar.so")
+
+STAR_OK = 0
+STAR_ERR_NULL_POINTER = 1
+STAR_ERR_INVALID_ARG = 2
+STAR_ERR_BAD_SCHEDULE = 3
+STAR_ERR_UNSUPPORTED = 4
+STAR_ERR_WORKSPACE_TOO_SMALL = 5
+STAR_ERR_CUDA = 6
+
+STAR_DTYPE_F32 = 0
+STAR_DTYPE_BF16 = 1
+STAR_MAX_WORKERS = 64
+
+
+class StarError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = _lib.star_status_string(status).decode()
+        extra = ""
+        if status == STAR_ERR_CUDA:
+            extra = " (cudaError %d)" % _lib.star_last_cuda_error()
+        super().__init__("%s failed: %s%s" % (where, name, extra))
+
+
+class star_multi_plan_t(ctypes.Structure):
+    _fields_ = [
+        ("magic", ctypes.c_uint64),
+        ("d_workspace", ctypes.c_void_p),
+        ("total_elements", ctypes.c_int64),
+        ("n_tiles", ctypes.c_int64),
+        ("complete_workers", ctypes.c_uint64),
+        ("n_tensors", ctypes.c_int32),
+        ("W", ctypes.c_int32),
+        ("grad_dtype", ctypes.c_int32),
+        ("tile_elements", ctypes.c_int32),
+    ]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "%s is missing: build it with `python -m paper_2512_09685_b200.build` "
+            "(there is no CPU fallback)" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    c_int, c_i64, c_vp, c_f = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float
+    lib.star_status_string.argtypes = [c_int]
+    lib.star_status_string.restype = ctypes.c_char_p
+    lib.star_last_cuda_error.argtypes = []
+    lib.star_last_cuda_error.restype = c_int
+    lib.star_launch_count.argtypes = []
+    lib.star_launch_count.restype = c_i64
+    lib.star_schedule_validate.argtypes = [c_vp, c_vp, c_int, c_int]
+    lib.star_schedule_static_x.argtypes = [c_vp, c_int, c_int, c_int, c_int, c_vp, c_vp, c_vp]
+    lib.star_schedule_from_labels.argtypes = [c_vp, c_int, c_vp, c_vp, c_vp]
+    lib.star_schedule_dynamic_x.argtypes = [c_vp, c_vp, c_int, c_vp, c_vp, c_vp]
+    lib.star_group_update.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
+                                      c_f, c_f, c_f, c_vp]
+    lib.star_multi_workspace_bytes.argtypes = [c_int, c_vp, c_int, c_vp]
+    lib.star_multi_prepare.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp,
+                                       ctypes.c_size_t, c_vp, c_vp]
+    lib.star_group_update_multi.argtypes = [c_vp, c_vp, c_vp, c_int, c_f, c_f, c_f, c_vp]
+    for name in ("star_schedule_validate", "star_schedule_static_x", "star_schedule_from_labels",
+                 "star_schedule_dynamic_x", "star_group_update", "star_multi_workspace_bytes",
+                 "star_multi_prepare", "star_group_update_multi"):
+        getattr(lib, name).restype = c_int
+    return lib
+
+
+_lib = _load()
+
+
+def _check(status: int, where: str) -> None:
+    if status != STAR_OK:
+        raise StarError(status, where)
+
+
+def _i32(values: Sequence[int]):
+    return (ctypes.c_int32 * max(len(values), 1))(*values)
+
+
+def star_status_string(status: int) -> str:
+    return _lib.star_status_string(status).decode()
+
+
+def star_last_cuda_error() -> int:
+    return _lib.star_last_cuda_error()
+
+
+def star_launch_count() -> int:
+    return _lib.star_launch_count()
+
+
+# ---------------------------------------------------------------------------
+# schedule encoding (host only)
+# ---------------------------------------------------------------------------
+Schedule = Tuple[List[int], List[int]]
+
+
+def _unpack(offsets, members, n_groups) -> Schedule:
+    K = n_groups.value
+    off = list(offsets[: K + 1])
+    return off, list(members[: off[K]])
+
+
+def star_schedule_validate(group_offsets: Sequence[int], group_members: Sequence[int],
+                           n_groups: int, W: int) -> int:
+    """Returns the status code (does not raise)."""
+    return _lib.star_schedule_validate(_i32(group_offsets), _i32(group_members), n_groups, W)
+
+
+def star_schedule_static_x(arrival_order: Optional[Sequence[int]], W: int, x: int,
+                           sort_members: bool = False) -> Schedule:
+    offsets, members, K = _i32([0] * (W + 1)), _i32([0] * W), ctypes.c_int(0)
+    if arrival_order is None:
+        order, n_arrived = None, W
+    else:
+        if len(arrival_order) > W:
+            raise StarError(STAR_ERR_INVALID_ARG, "star_schedule_static_x")
+        order, n_arrived = _i32(arrival_order), len(arrival_order)
+    _check(_lib.star_schedule_static_x(order, n_arrived, W, x, int(sort_members), offsets, members,
+                                       ctypes.byref(K)), "star_schedule_static_x")
+    return _unpack(offsets, members, K)
+
+
+def star_schedule_from_labels(group_of_worker: Sequence[int]) -> Schedule:
+    W = len(group_of_worker)
+    offsets, members, K = _i32([0] * (W + 1)), _i32([0] * W), ctypes.c_int(0)
+    _check(_lib.star_schedule_from_labels(_i32(group_of_worker), W, offsets, members,
+                                          ctypes.byref(K)), "star_schedule_from_labels")
+    return _unpack(offsets, members, K)
+
+
+def star_schedule_dynamic_x(iter_time: Sequence[float], cluster_of_worker: Sequence[int]) -> Schedule:
+    W = len(cluster_of_worker)
+    if len(iter_time) != W:
+        raise StarError(STAR_ERR_INVALID_ARG, "star_schedule_dynamic_x")
+    offsets, members, K = _i32([0] * (W + 1)), _i32([0] * W), ctypes.c_int(0)
+    times = (ctypes.c_double * max(W, 1))(*iter_time)
+    _check(_lib.star_schedule_dynamic_x(times, _i32(cluster_of_worker), W, offsets, members,
+                                        ctypes.byref(K)), "star_schedule_dynamic_x")
+    return _unpack(offsets, members, K)
+
+
+def encode(decision: ModeDecision) -> Schedule:
+    """Dispatch a mode decision to the matching C encoder."""
+    if decision.kind == "labels":
+        return star_schedule_from_labels(decision.labels)
+    if decision.kind == "static_x":
+        return star_schedule_static_x(decision.arrival_order, decision.W, decision.x,
+                                      decision.sort_members)
+    if decision.kind == "dynamic_x":
+        return star_schedule_dynamic_x(decision.iter_time, decision.labels)
+    raise ValueError(decision.kind)
+
+
+# ---------------------------------------------------------------------------
+# fused grouped update
+# ---------------------------------------------------------------------------
+def _grad_dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return STAR_DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return STAR_DTYPE_BF16
+    raise TypeError("gradients must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _state(t: torch.Tensor, what: str) -> int:
+    if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous():
+        raise TypeError("%s must be a contiguous float32 CUDA tensor" % what)
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def star_group_update(params: torch.Tensor, momentum: torch.Tensor,
+                      grads: Sequence[Optional[torch.Tensor]], group_offsets: Sequence[int],
+                      group_members: Sequence[int], lr: float, mu: float, wd: float,
+                      stream=None) -> None:
+    """In-place fused grouped update of one flat tensor on the current device."""
+    n = params.numel()
+    p, v = _state(params, "params"), _state(momentum, "momentum")
+    if momentum.numel() != n:
+        raise ValueError("params and momentum differ in size")
+    W = len(grads)
+    ptrs = (ctypes.c_void_p * max(W, 1))()
+    dt = None
+    for w, g in enumerate(grads):
+        if g is None:
+            continue
+        if not g.is_cuda or not g.is_contiguous() or g.numel() != n:
+            raise ValueError("gradient %d must be a contiguous CUDA tensor of %d elements" % (w, n))
+        d = _grad_dtype(g)
+        if dt is not None and d != dt:
+            raise TypeError("gradients differ in dtype")
+        dt = d
+        ptrs[w] = g.data_ptr()
+    K = len(group_offsets) - 1 if len(group_offsets) else 0
+    _check(_lib.star_group_update(p, v, ptrs, W, STAR_DTYPE_F32 if dt is None else dt, n,
+                                  _i32(group_offsets), _i32(group_members), K, lr, mu, wd,
+                                  _stream(stream)), "star_group_update")
+
+
+def star_multi_workspace_bytes(sizes: Sequence[int], W: int) -> int:
+    out = ctypes.c_size_t(0)
+    arr = (ctypes.c_int64 * max(len(sizes), 1))(*sizes)
+    _check(_lib.star_multi_workspace_bytes(len(sizes), arr, W, ctypes.byref(out)),
+           "star_multi_workspace_bytes")
+    return out.value
+
+
+def star_multi_prepare(params: Sequence[torch.Tensor], momentum: Sequence[torch.Tensor],
+                       grads: Sequence[Sequence[Optional[torch.Tensor]]], workspace: torch.Tensor,
+                       stream=None) -> star_multi_plan_t:
+    """``grads[w][t]`` = worker w's gradient for tensor t.  ``workspace`` is a
+    uint8 CUDA tensor of at least :func:`star_multi_workspace_bytes` bytes; the
+    returned plan refers to it (keep the tensor alive)."""
+    T, W = len(params), len(grads)
+    if len(momentum) != T or any(len(g) != T for g in grads):
+        raise ValueError("params, momentum and every worker's gradient list need one entry per tensor")
+    sizes = [p.numel() for p in params]
+    P = (ctypes.c_void_p * max(T, 1))(*[_state(p, "params") if p.numel() else None for p in params])
+    V = (ctypes.c_void_p * max(T, 1))(*[_state(v, "momentum") if v.numel() else None for v in momentum])
+    G = (ctypes.c_void_p * max(T * W, 1))()
+    dt = None
+    for w in range(W):
+        for t in range(T):
+            g = grads[w][t]
+            if g is None:
+                continue
+            if not g.is_cuda or not g.is_contiguous() or g.numel() != sizes[t]:
+                raise ValueError("gradient [%d][%d] must be a contiguous CUDA tensor of %d elements"
+                                 % (w, t, sizes[t]))
+            d = _grad_dtype(g)
+            if dt is not None and d != dt:
+                raise TypeError("gradients differ in dtype")
+            dt = d
+            G[t * W + w] = g.data_ptr() if sizes[t] else None
+    if momentum and any(v.numel() != s for v, s in zip(momentum, sizes)):
+        raise ValueError("params and momentum differ in size")
+    if workspace.dtype != torch.uint8 or not workspace.is_cuda or not workspace.is_contiguous():
+        raise TypeError("workspace must be a contiguous uint8 CUDA tensor")
+    plan = star_multi_plan_t()
+    S = (ctypes.c_int64 * max(T, 1))(*sizes)
+    _check(_lib.star_multi_prepare(T, P, V, G, S, W, STAR_DTYPE_F32 if dt is None else dt,
+                                   workspace.data_ptr(), workspace.numel(), _stream(stream),
+                                   ctypes.byref(plan)), "star_multi_prepare")
+    return plan
+
+
+def star_group_update_multi(plan: star_multi_plan_t, group_offsets: Sequence[int],
+                            group_members: Sequence[int], lr: float, mu: float, wd: float,
+                            stream=None) -> None:
+    K = len(group_offsets) - 1 if len(group_offsets) else 0
+    _check(_lib.star_group_update_multi(ctypes.byref(plan), _i32(group_offsets), _i32(group_members),
+                                        K, lr, mu, wd, _stream(stream)), "star_group_update_multi")

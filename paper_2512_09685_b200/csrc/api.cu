@@ -1,0 +1,361 @@
+// C-ABI entry points: argument checks on the host, then one kernel launch.
+#include <atomic>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "kernels.cuh"
+#include "star.h"
+
+namespace {
+
+using namespace star;
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<int64_t> g_launches{0};
+
+star_status_t cuda_failed(cudaError_t e)
+{
+    g_last_cuda_error = static_cast<int>(e);
+    return STAR_ERR_CUDA;
+}
+
+constexpr uint64_t kPlanMagic = 0x53544152504c414eull;   // "STARPLAN"
+constexpr size_t kWorkspaceAlign = 256;
+
+// ---------------------------------------------------------------------------
+// Launch geometry: a persistent grid of (SM count x resident blocks) blocks,
+// capped by the work there is.  Queried once per device and kernel.
+// ---------------------------------------------------------------------------
+constexpr int kMaxDevices = 64;
+
+struct Geometry {
+    std::atomic<int> blocks{0};
+};
+
+template <typename Kernel>
+cudaError_t resident_blocks(Kernel kernel, Geometry *cache, int *blocks_out)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    int blocks = cache[dev].blocks.load(std::memory_order_relaxed);
+    if (blocks == 0) {
+        int sms = 0, per_sm = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlockThreads, 0);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) per_sm = 1;
+        blocks = sms * per_sm;
+        cache[dev].blocks.store(blocks, std::memory_order_relaxed);
+    }
+    *blocks_out = blocks;
+    return cudaSuccess;
+}
+
+// ---------------------------------------------------------------------------
+// Schedule: validate, then flatten into the kernel's slot list.
+// ---------------------------------------------------------------------------
+star_status_t flatten_schedule(const int32_t *group_offsets, const int32_t *group_members, int n_groups,
+                               int W, float lr, FlatSchedule *out)
+{
+    const star_status_t st = star_schedule_validate(group_offsets, group_members, n_groups, W);
+    if (st != STAR_OK) return st;
+    std::memset(out, 0, sizeof *out);
+    out->n_slots = n_groups > 0 ? group_offsets[n_groups] : 0;
+    for (int k = 0; k < n_groups; ++k) {
+        const int first = group_offsets[k], last = group_offsets[k + 1];
+        for (int j = first; j < last; ++j) out->member[j] = static_cast<uint8_t>(group_members[j]);
+        out->group_size[last - 1] = static_cast<uint8_t>(last - first);
+        out->neg_lr[last - 1] = -lr;
+    }
+    return STAR_OK;
+}
+
+bool overlaps(const void *a, size_t a_bytes, const void *b, size_t b_bytes)
+{
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
+}
+
+bool aligned(const void *p, size_t bytes) { return reinterpret_cast<uintptr_t>(p) % bytes == 0; }
+
+// Kernel choices.  bf16: 16 elements per thread (one 32-byte gradient load per
+// worker, 64 bytes each of p and v); fp32: 8 elements per thread.
+constexpr int kVecBF16 = 16;
+constexpr int kVecF32 = 8;
+constexpr int kDepthVector = 8;
+constexpr int kDepthScalar = 8;
+constexpr int kVectorBytes = 32;          // base alignment the vector path needs
+constexpr int kMultiVecPerThread = 1;
+
+template <typename G, int VEC>
+star_status_t launch_flat(const FlatArgs &args, cudaStream_t stream)
+{
+    static Geometry cache[kMaxDevices];
+    constexpr int depth = VEC == 1 ? kDepthScalar : kDepthVector;
+    auto kernel = star_update_flat_kernel<G, VEC, depth>;
+    int blocks = 0;
+    cudaError_t e = resident_blocks(kernel, cache, &blocks);
+    if (e != cudaSuccess) return cuda_failed(e);
+    const int64_t work = (args.n / VEC + kBlockThreads - 1) / kBlockThreads;
+    const int grid = static_cast<int>(work < 1 ? 1 : (work < blocks ? work : blocks));
+    kernel<<<grid, kBlockThreads, 0, stream>>>(args);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return STAR_OK;
+}
+
+}  // namespace
+
+extern "C" const char *star_status_string(star_status_t status)
+{
+    switch (status) {
+    case STAR_OK: return "STAR_OK";
+    case STAR_ERR_NULL_POINTER: return "STAR_ERR_NULL_POINTER";
+    case STAR_ERR_INVALID_ARG: return "STAR_ERR_INVALID_ARG";
+    case STAR_ERR_BAD_SCHEDULE: return "STAR_ERR_BAD_SCHEDULE";
+    case STAR_ERR_UNSUPPORTED: return "STAR_ERR_UNSUPPORTED";
+    case STAR_ERR_WORKSPACE_TOO_SMALL: return "STAR_ERR_WORKSPACE_TOO_SMALL";
+    case STAR_ERR_CUDA: return "STAR_ERR_CUDA";
+    }
+    return "STAR_ERR_UNKNOWN";
+}
+
+extern "C" int star_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" int64_t star_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+extern "C" star_status_t star_group_update(float *params, float *momentum, const void *const *grads, int W,
+                                           star_dtype_t grad_dtype, int64_t n,
+                                           const int32_t *group_offsets, const int32_t *group_members,
+                                           int n_groups, float lr, float mu, float wd, void *cuda_stream)
+{
+    if (n < 0 || W < 0) return STAR_ERR_INVALID_ARG;
+    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    FlatArgs args;
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, lr, &args.sched);
+    if (st != STAR_OK) return st;
+    if (n == 0 || n_groups == 0) return STAR_OK;
+    if (!params || !momentum || !grads) return STAR_ERR_NULL_POINTER;
+
+    const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
+    if (!aligned(params, 4) || !aligned(momentum, 4)) return STAR_ERR_INVALID_ARG;
+    if (overlaps(params, state_bytes, momentum, state_bytes)) return STAR_ERR_INVALID_ARG;
+    bool vector_ok = aligned(params, kVectorBytes) && aligned(momentum, kVectorBytes);
+    std::memset(args.grads, 0, sizeof args.grads);
+    for (int j = 0; j < args.sched.n_slots; ++j) {
+        const int w = args.sched.member[j];
+        const void *g = grads[w];
+        if (!g) return STAR_ERR_NULL_POINTER;
+        if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
+        if (overlaps(g, grad_bytes, params, state_bytes) || overlaps(g, grad_bytes, momentum, state_bytes))
+            return STAR_ERR_INVALID_ARG;
+        vector_ok = vector_ok && aligned(g, kVectorBytes);
+        args.grads[w] = g;
+    }
+    args.params = params;
+    args.momentum = momentum;
+    args.n = n;
+    args.hyper = Hyper{mu, wd};
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (grad_dtype == STAR_DTYPE_BF16)
+        return vector_ok ? launch_flat<GradBF16, kVecBF16>(args, stream) : launch_flat<GradBF16, 1>(args, stream);
+    return vector_ok ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
+}
+
+// ---------------------------------------------------------------------------
+// Tensor lists.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t tile_elements(star_dtype_t dt)
+{
+    return static_cast<int64_t>(kBlockThreads) * kMultiVecPerThread * (dt == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32);
+}
+
+// The workspace is sized for the smaller (fp32) tile, i.e. the larger tile
+// count, so that its size does not depend on the gradient dtype.
+constexpr int64_t kTileForSizing = static_cast<int64_t>(kBlockThreads) * kMultiVecPerThread * kVecF32;
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WorkspaceLayout {
+    size_t tensors_off, grads_off, tiles_off, total;
+};
+
+WorkspaceLayout layout_for(int n_tensors, int W, int64_t n_tiles)
+{
+    WorkspaceLayout l;
+    l.tensors_off = 0;
+    l.grads_off = round_up(l.tensors_off + sizeof(TensorEntry) * static_cast<size_t>(n_tensors), kWorkspaceAlign);
+    l.tiles_off = round_up(l.grads_off + sizeof(void *) * static_cast<size_t>(n_tensors) * static_cast<size_t>(W),
+                           kWorkspaceAlign);
+    l.total = round_up(l.tiles_off + sizeof(int32_t) * static_cast<size_t>(n_tiles), kWorkspaceAlign);
+    if (l.total == 0) l.total = kWorkspaceAlign;
+    return l;
+}
+
+star_status_t count_tiles(int n_tensors, const int64_t *sizes, int64_t tile, int64_t *n_tiles, int64_t *total)
+{
+    *n_tiles = 0;
+    *total = 0;
+    for (int t = 0; t < n_tensors; ++t) {
+        if (sizes[t] < 0) return STAR_ERR_INVALID_ARG;
+        *n_tiles += (sizes[t] + tile - 1) / tile;
+        *total += sizes[t];
+    }
+    return STAR_OK;
+}
+
+template <typename G, int VEC>
+star_status_t launch_multi(const MultiArgs &args, cudaStream_t stream)
+{
+    static Geometry cache[kMaxDevices];
+    auto kernel = star_update_multi_kernel<G, VEC, kDepthVector, kMultiVecPerThread>;
+    int blocks = 0;
+    cudaError_t e = resident_blocks(kernel, cache, &blocks);
+    if (e != cudaSuccess) return cuda_failed(e);
+    const int grid = static_cast<int>(args.n_tiles < blocks ? args.n_tiles : blocks);
+    kernel<<<grid, kBlockThreads, 0, stream>>>(args);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return STAR_OK;
+}
+
+}  // namespace
+
+extern "C" star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *sizes, int W,
+                                                    size_t *bytes_out)
+{
+    if (!bytes_out) return STAR_ERR_NULL_POINTER;
+    if (n_tensors < 0 || W < 0) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    if (n_tensors > 0 && !sizes) return STAR_ERR_NULL_POINTER;
+    int64_t n_tiles = 0, total = 0;
+    const star_status_t st = count_tiles(n_tensors, sizes, kTileForSizing, &n_tiles, &total);
+    if (st != STAR_OK) return st;
+    *bytes_out = layout_for(n_tensors, W, n_tiles).total;
+    return STAR_OK;
+}
+
+extern "C" star_status_t star_multi_prepare(int n_tensors, float *const *params, float *const *momentum,
+                                            const void *const *grads, const int64_t *sizes, int W,
+                                            star_dtype_t grad_dtype, void *d_workspace,
+                                            size_t workspace_bytes, void *cuda_stream,
+                                            star_multi_plan_t *plan_out)
+{
+    if (!plan_out) return STAR_ERR_NULL_POINTER;
+    std::memset(plan_out, 0, sizeof *plan_out);
+    if (n_tensors < 0 || W < 0) return STAR_ERR_INVALID_ARG;
+    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    if (n_tensors > 0 && (!params || !momentum || !grads || !sizes)) return STAR_ERR_NULL_POINTER;
+    if (!d_workspace) return STAR_ERR_NULL_POINTER;
+    if (!aligned(d_workspace, kWorkspaceAlign)) return STAR_ERR_INVALID_ARG;
+
+    const int64_t tile = tile_elements(grad_dtype);
+    int64_t n_tiles = 0, total = 0, sizing_tiles = 0, unused = 0;
+    star_status_t st = count_tiles(n_tensors, sizes, tile, &n_tiles, &total);
+    if (st != STAR_OK) return st;
+    count_tiles(n_tensors, sizes, kTileForSizing, &sizing_tiles, &unused);
+    const WorkspaceLayout need = layout_for(n_tensors, W, sizing_tiles);
+    if (workspace_bytes < need.total) return STAR_ERR_WORKSPACE_TOO_SMALL;
+    const WorkspaceLayout l = layout_for(n_tensors, W, n_tiles);
+
+    const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    uint64_t complete = W == 64 ? ~uint64_t{0} : ((uint64_t{1} << W) - 1);
+    std::vector<unsigned char> host(l.total, 0);
+    TensorEntry *entries = reinterpret_cast<TensorEntry *>(host.data() + l.tensors_off);
+    const void **table = reinterpret_cast<const void **>(host.data() + l.grads_off);
+    int32_t *tile_tensor = reinterpret_cast<int32_t *>(host.data() + l.tiles_off);
+    int64_t next_tile = 0;
+    for (int t = 0; t < n_tensors; ++t) {
+        const int64_t size = sizes[t];
+        TensorEntry &e = entries[t];
+        e.params = params[t];
+        e.momentum = momentum[t];
+        e.size = size;
+        e.first_tile = next_tile;
+        e.pad = 0;
+        bool vector_ok = true;
+        if (size > 0) {
+            if (!params[t] || !momentum[t]) return STAR_ERR_NULL_POINTER;
+            if (!aligned(params[t], 4) || !aligned(momentum[t], 4)) return STAR_ERR_INVALID_ARG;
+            const size_t state_bytes = static_cast<size_t>(size) * 4;
+            if (overlaps(params[t], state_bytes, momentum[t], state_bytes)) return STAR_ERR_INVALID_ARG;
+            vector_ok = aligned(params[t], kVectorBytes) && aligned(momentum[t], kVectorBytes);
+        }
+        for (int w = 0; w < W; ++w) {
+            const void *g = grads[static_cast<size_t>(t) * W + w];
+            table[static_cast<size_t>(t) * W + w] = g;
+            if (size == 0) continue;
+            if (!g) {
+                complete &= ~(uint64_t{1} << w);
+                continue;
+            }
+            if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
+            const size_t state_bytes = static_cast<size_t>(size) * 4, grad_bytes = static_cast<size_t>(size) * gsize;
+            if (overlaps(g, grad_bytes, params[t], state_bytes) || overlaps(g, grad_bytes, momentum[t], state_bytes))
+                return STAR_ERR_INVALID_ARG;
+            vector_ok = vector_ok && aligned(g, kVectorBytes);
+        }
+        e.vector_ok = vector_ok ? 1 : 0;
+        const int64_t tiles_here = (size + tile - 1) / tile;
+        for (int64_t i = 0; i < tiles_here; ++i) tile_tensor[next_tile + i] = t;
+        next_tile += tiles_here;
+    }
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const cudaError_t e = cudaMemcpyAsync(d_workspace, host.data(), l.total, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_failed(e);
+
+    plan_out->magic = kPlanMagic;
+    plan_out->d_workspace = d_workspace;
+    plan_out->total_elements = total;
+    plan_out->n_tiles = n_tiles;
+    plan_out->complete_workers = complete;
+    plan_out->n_tensors = n_tensors;
+    plan_out->W = W;
+    plan_out->grad_dtype = static_cast<int32_t>(grad_dtype);
+    plan_out->tile_elements = static_cast<int32_t>(tile);
+    return STAR_OK;
+}
+
+extern "C" star_status_t star_group_update_multi(const star_multi_plan_t *plan,
+                                                 const int32_t *group_offsets, const int32_t *group_members,
+                                                 int n_groups, float lr, float mu, float wd,
+                                                 void *cuda_stream)
+{
+    if (!plan) return STAR_ERR_NULL_POINTER;
+    if (plan->magic != kPlanMagic || !plan->d_workspace) return STAR_ERR_INVALID_ARG;
+    MultiArgs args;
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, plan->W, lr, &args.sched);
+    if (st != STAR_OK) return st;
+    if (plan->n_tiles == 0 || n_groups == 0) return STAR_OK;
+    for (int j = 0; j < args.sched.n_slots; ++j)
+        if (!(plan->complete_workers >> args.sched.member[j] & 1u)) return STAR_ERR_NULL_POINTER;
+
+    const star_dtype_t dt = static_cast<star_dtype_t>(plan->grad_dtype);
+    const int64_t sizing_tiles = plan->n_tiles;     // layout offsets depend on n_tensors and W only up to tiles_off
+    const WorkspaceLayout l = layout_for(plan->n_tensors, plan->W, sizing_tiles);
+    const char *base = static_cast<const char *>(plan->d_workspace);
+    args.tensors = reinterpret_cast<const TensorEntry *>(base + l.tensors_off);
+    args.grads = reinterpret_cast<const void *const *>(base + l.grads_off);
+    args.tile_tensor = reinterpret_cast<const int32_t *>(base + l.tiles_off);
+    args.n_tiles = plan->n_tiles;
+    args.W = plan->W;
+    args.hyper = Hyper{mu, wd};
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (dt == STAR_DTYPE_BF16) return launch_multi<GradBF16, kVecBF16>(args, stream);
+    if (dt == STAR_DTYPE_F32) return launch_multi<GradF32, kVecF32>(args, stream);
+    return STAR_ERR_INVALID_ARG;
+}

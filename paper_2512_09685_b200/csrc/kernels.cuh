@@ -1,0 +1,316 @@
+// Device code of the fused grouped update (sm_100a).
+//
+// One thread owns VEC consecutive elements of one tensor.  It loads p and v,
+// then walks the flattened schedule (all members of all groups, in order) in
+// chunks of DEPTH members: the DEPTH gradient loads of a chunk are issued back
+// to back before any of them is consumed, so each thread keeps
+// DEPTH * 16..32 bytes in flight on top of p and v.  Every group's update is
+// applied in registers; p and v are stored once.
+//
+// The arithmetic is the pinned binary32 sequence
+//     s = g_0 + g_1 + ... ; gbar = s / |G| ; d = fma(wd, p, gbar) ;
+//     v = fma(mu, v, d)   ; p = fma(-lr, v, p)
+// written with round-to-nearest intrinsics, which the compiler neither
+// contracts nor reassociates.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace star {
+
+constexpr int kMaxWorkers = 64;
+constexpr int kBlockThreads = 256;
+
+// The schedule as the kernel sees it: one slot per scheduled worker, in the
+// order the gradients are consumed.  A slot that closes a group carries that
+// group's size and (negated) learning rate.
+struct FlatSchedule {
+    int32_t n_slots;
+    uint8_t member[kMaxWorkers];       // slot -> worker index
+    uint8_t group_size[kMaxWorkers];   // |G_k| on the last slot of group k, else 0
+    float neg_lr[kMaxWorkers];         // -lr_k on the last slot of group k
+};
+
+struct Hyper {
+    float mu;
+    float wd;
+};
+
+// ---------------------------------------------------------------------------
+// Memory operations.  Gradients are read exactly once: non-coherent path, no
+// L1 allocation.  p and v are read once and written once.
+// ---------------------------------------------------------------------------
+template <int BYTES> struct Raw;              // BYTES of payload in 32-bit registers
+template <> struct Raw<2>  { uint32_t w[1]; };
+template <> struct Raw<4>  { uint32_t w[1]; };
+template <> struct Raw<16> { uint32_t w[4]; };
+template <> struct Raw<32> { uint32_t w[8]; };
+
+template <int BYTES> __device__ __forceinline__ Raw<BYTES> load_stream(const void *p);
+
+template <> __device__ __forceinline__ Raw<2> load_stream<2>(const void *p)
+{
+    Raw<2> r;
+    unsigned short h;
+    asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(h) : "l"(p));
+    r.w[0] = h;
+    return r;
+}
+template <> __device__ __forceinline__ Raw<4> load_stream<4>(const void *p)
+{
+    Raw<4> r;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(r.w[0]) : "l"(p));
+    return r;
+}
+template <> __device__ __forceinline__ Raw<16> load_stream<16>(const void *p)
+{
+    Raw<16> r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p));
+    return r;
+}
+template <> __device__ __forceinline__ Raw<32> load_stream<32>(const void *p)
+{
+    Raw<32> r;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]),
+                   "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7]) : "l"(p));
+    return r;
+}
+
+// p / v: VEC floats, through 4-, 16- or 32-byte accesses.
+template <int VEC> __device__ __forceinline__ void load_state(const float *src, float (&x)[VEC])
+{
+    if constexpr (VEC == 1) {
+        x[0] = *src;
+    } else if constexpr (VEC % 8 == 0) {
+#pragma unroll
+        for (int q = 0; q < VEC / 8; ++q) {
+            uint32_t w[8];
+            asm volatile("ld.global.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]),
+                           "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "l"(src + 8 * q));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) x[8 * q + e] = __uint_as_float(w[e]);
+        }
+    } else {
+#pragma unroll
+        for (int q = 0; q < VEC / 4; ++q) {
+            float4 t;
+            asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                         : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "l"(src + 4 * q));
+            x[4 * q + 0] = t.x; x[4 * q + 1] = t.y; x[4 * q + 2] = t.z; x[4 * q + 3] = t.w;
+        }
+    }
+}
+
+template <int VEC> __device__ __forceinline__ void store_state(float *dst, const float (&x)[VEC])
+{
+    if constexpr (VEC == 1) {
+        *dst = x[0];
+    } else if constexpr (VEC % 8 == 0) {
+#pragma unroll
+        for (int q = 0; q < VEC / 8; ++q) {
+            asm volatile("st.global.L1::no_allocate.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                         :: "r"(__float_as_uint(x[8 * q + 0])), "r"(__float_as_uint(x[8 * q + 1])),
+                            "r"(__float_as_uint(x[8 * q + 2])), "r"(__float_as_uint(x[8 * q + 3])),
+                            "r"(__float_as_uint(x[8 * q + 4])), "r"(__float_as_uint(x[8 * q + 5])),
+                            "r"(__float_as_uint(x[8 * q + 6])), "r"(__float_as_uint(x[8 * q + 7])),
+                            "l"(dst + 8 * q) : "memory");
+        }
+    } else {
+#pragma unroll
+        for (int q = 0; q < VEC / 4; ++q) {
+            asm volatile("st.global.L1::no_allocate.v4.f32 [%4], {%0,%1,%2,%3};"
+                         :: "f"(x[4 * q + 0]), "f"(x[4 * q + 1]), "f"(x[4 * q + 2]),
+                            "f"(x[4 * q + 3]), "l"(dst + 4 * q) : "memory");
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Gradient element types.
+// ---------------------------------------------------------------------------
+struct GradF32 {
+    static constexpr int kBytes = 4;
+    template <int VEC> static __device__ __forceinline__ void widen(const Raw<VEC * 4> &r, float (&f)[VEC])
+    {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) f[e] = __uint_as_float(r.w[e]);
+    }
+};
+
+struct GradBF16 {
+    static constexpr int kBytes = 2;
+    // bf16 is the upper half of a binary32: widening is a shift / a mask.
+    template <int VEC> static __device__ __forceinline__ void widen(const Raw<VEC * 2> &r, float (&f)[VEC])
+    {
+        if constexpr (VEC == 1) {
+            f[0] = __uint_as_float(r.w[0] << 16);
+        } else {
+#pragma unroll
+            for (int e = 0; e < VEC / 2; ++e) {
+                f[2 * e + 0] = __uint_as_float(r.w[e] << 16);
+                f[2 * e + 1] = __uint_as_float(r.w[e] & 0xffff0000u);
+            }
+        }
+    }
+};
+
+// One group update on VEC elements.
+template <int VEC>
+__device__ __forceinline__ void apply_update(float (&p)[VEC], float (&v)[VEC], const float (&gbar)[VEC],
+                                             float neg_lr, const Hyper &h)
+{
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        const float d = __fmaf_rn(h.wd, p[e], gbar[e]);
+        v[e] = __fmaf_rn(h.mu, v[e], d);
+        p[e] = __fmaf_rn(neg_lr, v[e], p[e]);
+    }
+}
+
+// All groups of the round on the VEC elements starting at element `first` of
+// one tensor.  grad_ptr(slot) returns the base pointer of the slot's worker.
+template <typename G, int VEC, int DEPTH, typename GradPtr>
+__device__ __forceinline__ void update_vector(float *__restrict__ params, float *__restrict__ momentum,
+                                              int64_t first, const FlatSchedule &s, const Hyper &h,
+                                              GradPtr grad_ptr)
+{
+    constexpr int GB = VEC * G::kBytes;
+    float p[VEC], v[VEC], sum[VEC];
+    load_state<VEC>(params + first, p);
+    load_state<VEC>(momentum + first, v);
+    // -0.0f is the additive identity of IEEE addition (x + -0 == x for every x,
+    // including x == -0), so a running sum started there equals the plain
+    // left-to-right sum that starts at the first member.
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) sum[e] = -0.0f;
+
+    const int n_slots = s.n_slots;
+    for (int base = 0; base < n_slots; base += DEPTH) {
+        Raw<GB> raw[DEPTH];
+#pragma unroll
+        for (int j = 0; j < DEPTH; ++j) {
+            if (base + j < n_slots) {
+                const char *g = static_cast<const char *>(grad_ptr(base + j));
+                raw[j] = load_stream<GB>(g + first * G::kBytes);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < DEPTH; ++j) {
+            if (base + j < n_slots) {
+                float f[VEC];
+                G::template widen<VEC>(raw[j], f);
+                const int gs = s.group_size[base + j];
+                if (gs == 1) {                       // singleton group: the mean is the gradient
+                    apply_update<VEC>(p, v, f, s.neg_lr[base + j], h);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) sum[e] = __fadd_rn(sum[e], f[e]);
+                    if (gs != 0) {
+                        const float count = static_cast<float>(gs);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) sum[e] = __fdiv_rn(sum[e], count);
+                        apply_update<VEC>(p, v, sum, s.neg_lr[base + j], h);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) sum[e] = -0.0f;
+                    }
+                }
+            }
+        }
+    }
+    store_state<VEC>(params + first, p);
+    store_state<VEC>(momentum + first, v);
+}
+
+// ---------------------------------------------------------------------------
+// Single flat tensor.
+// ---------------------------------------------------------------------------
+struct FlatArgs {
+    float *params;
+    float *momentum;
+    const void *grads[kMaxWorkers];
+    int64_t n;
+    FlatSchedule sched;
+    Hyper hyper;
+};
+
+// Vector kernel: requires 16-byte (VEC*kBytes == 16) or 32-byte aligned bases.
+// Grid-stride over vectors; the last < VEC elements are done one by one by the
+// first threads of block 0.
+template <typename G, int VEC, int DEPTH>
+__global__ void __launch_bounds__(kBlockThreads)
+star_update_flat_kernel(const __grid_constant__ FlatArgs a)
+{
+    const int64_t n_vec = a.n / VEC;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlockThreads;
+    auto grad_ptr = [&](int slot) -> const void * { return a.grads[a.sched.member[slot]]; };
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kBlockThreads + threadIdx.x; i < n_vec; i += stride)
+        update_vector<G, VEC, DEPTH>(a.params, a.momentum, i * VEC, a.sched, a.hyper, grad_ptr);
+    if constexpr (VEC > 1) {
+        const int64_t tail = n_vec * VEC + threadIdx.x;
+        if (blockIdx.x == 0 && threadIdx.x < VEC && tail < a.n)
+            update_vector<G, 1, DEPTH>(a.params, a.momentum, tail, a.sched, a.hyper, grad_ptr);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Tensor list.  The device workspace holds, in this order (each array 256-byte
+// aligned): per-tensor TensorEntry records, the gradient pointer table
+// [n_tensors * W], and tile_tensor[n_tiles] (tile -> tensor index).  Tiles of a
+// tensor are consecutive; TensorEntry::first_tile is the tensor's first tile.
+// ---------------------------------------------------------------------------
+struct TensorEntry {
+    float *params;
+    float *momentum;
+    int64_t size;          // elements
+    int64_t first_tile;
+    int32_t vector_ok;     // all of the tensor's buffers are aligned for the vector path
+    int32_t pad;
+};
+
+struct MultiArgs {
+    const TensorEntry *tensors;
+    const void *const *grads;       // [n_tensors * W]
+    const int32_t *tile_tensor;     // [n_tiles]
+    int64_t n_tiles;
+    int32_t W;
+    FlatSchedule sched;
+    Hyper hyper;
+};
+
+template <typename G, int VEC, int DEPTH, int VEC_PER_THREAD>
+__global__ void __launch_bounds__(kBlockThreads)
+star_update_multi_kernel(const __grid_constant__ MultiArgs a)
+{
+    constexpr int64_t kTile = static_cast<int64_t>(kBlockThreads) * VEC * VEC_PER_THREAD;
+    for (int64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
+        const int32_t t = __ldg(a.tile_tensor + tile);
+        const TensorEntry te = a.tensors[t];
+        const unsigned long long *row =
+            reinterpret_cast<const unsigned long long *>(a.grads) + static_cast<int64_t>(t) * a.W;
+        auto grad_ptr = [&](int slot) -> const void * {
+            return reinterpret_cast<const void *>(__ldg(row + a.sched.member[slot]));
+        };
+        const int64_t begin = (tile - te.first_tile) * kTile;
+        const int64_t end = min(te.size, begin + kTile);
+        if (te.vector_ok) {
+            const int64_t vec_end = begin + (end - begin) / VEC * VEC;
+#pragma unroll 1
+            for (int64_t i = begin + static_cast<int64_t>(threadIdx.x) * VEC; i < vec_end;
+                 i += static_cast<int64_t>(kBlockThreads) * VEC)
+                update_vector<G, VEC, DEPTH>(te.params, te.momentum, i, a.sched, a.hyper, grad_ptr);
+            if (vec_end + threadIdx.x < end)         // fewer than VEC leftovers
+                update_vector<G, 1, DEPTH>(te.params, te.momentum, vec_end + threadIdx.x, a.sched,
+                                           a.hyper, grad_ptr);
+        } else {
+#pragma unroll 1
+            for (int64_t i = begin + threadIdx.x; i < end; i += kBlockThreads)
+                update_vector<G, 1, DEPTH>(te.params, te.momentum, i, a.sched, a.hyper, grad_ptr);
+        }
+    }
+}
+
+}  // namespace star
