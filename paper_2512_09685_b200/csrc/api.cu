@@ -84,14 +84,14 @@ bool overlaps(const void *a, size_t a_bytes, const void *b, size_t b_bytes)
 
 bool aligned(const void *p, size_t bytes) { return reinterpret_cast<uintptr_t>(p) % bytes == 0; }
 
-// Kernel choices.  bf16: 16 elements per thread (one 32-byte gradient load per
-// worker, 64 bytes each of p and v); fp32: 8 elements per thread.
-constexpr int kVecBF16 = 16;
-constexpr int kVecF32 = 8;
-constexpr int kDepthVector = 8;
-constexpr int kDepthScalar = 8;
+// Kernel choices.  bf16: 8 elements per thread (one 16-byte gradient load per
+// worker, 32 bytes each of p and v); fp32: 4 elements per thread; 4 gradient
+// loads in flight per thread.
+constexpr int kVecBF16 = 8;
+constexpr int kVecF32 = 4;
+constexpr int kDepthVector = 4;
+constexpr int kDepthScalar = 4;
 constexpr int kVectorBytes = 32;          // base alignment the vector path needs
-constexpr int kMultiVecPerThread = 1;
 
 template <typename G, int VEC>
 star_status_t launch_flat(const FlatArgs &args, cudaStream_t stream)
@@ -178,12 +178,12 @@ namespace {
 
 constexpr int64_t tile_elements(star_dtype_t dt)
 {
-    return static_cast<int64_t>(kBlockThreads) * kMultiVecPerThread * (dt == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32);
+    return static_cast<int64_t>(kBlockThreads) * (dt == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32);
 }
 
 // The workspace is sized for the smaller (fp32) tile, i.e. the larger tile
 // count, so that its size does not depend on the gradient dtype.
-constexpr int64_t kTileForSizing = static_cast<int64_t>(kBlockThreads) * kMultiVecPerThread * kVecF32;
+constexpr int64_t kTileForSizing = static_cast<int64_t>(kBlockThreads) * kVecF32;
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -219,7 +219,7 @@ template <typename G, int VEC>
 star_status_t launch_multi(const MultiArgs &args, cudaStream_t stream)
 {
     static Geometry cache[kMaxDevices];
-    auto kernel = star_update_multi_kernel<G, VEC, kDepthVector, kMultiVecPerThread>;
+    auto kernel = star_update_multi_kernel<G, VEC, kDepthVector>;
     int blocks = 0;
     cudaError_t e = resident_blocks(kernel, cache, &blocks);
     if (e != cudaSuccess) return cuda_failed(e);

@@ -21,6 +21,11 @@ namespace star {
 
 constexpr int kMaxWorkers = 64;
 constexpr int kBlockThreads = 256;
+// Resident blocks per SM the vector kernels are compiled for: 4 x 256 threads
+// at <= 64 registers.  Measured on B200: 32 resident warps per SM with 4 loads
+// in flight per thread reach the HBM copy rate; one block of 145-register
+// threads (deeper chunks, wider vectors) reached only 63 % of it.
+constexpr int kResidentBlocks = 4;
 
 // The schedule as the kernel sees it: one slot per scheduled worker, in the
 // order the gradients are consumed.  A slot that closes a group carries that
@@ -172,16 +177,18 @@ __device__ __forceinline__ void apply_update(float (&p)[VEC], float (&v)[VEC], c
 }
 
 // All groups of the round on the VEC elements starting at element `first` of
-// one tensor.  grad_ptr(slot) returns the base pointer of the slot's worker.
-template <typename G, int VEC, int DEPTH, typename GradPtr>
-__device__ __forceinline__ void update_vector(float *__restrict__ params, float *__restrict__ momentum,
-                                              int64_t first, const FlatSchedule &s, const Hyper &h,
-                                              GradPtr grad_ptr)
+// one tensor.  grad_ptr(slot) returns the base pointer of the slot's worker;
+// state_ptr(0) / state_ptr(1) return the tensor's params / momentum base and are
+// asked again at store time, so that a caller whose bases live in memory need
+// not hold them in registers across the update.
+template <typename G, int VEC, int DEPTH, typename StatePtr, typename GradPtr>
+__device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first, const FlatSchedule &s,
+                                              const Hyper &h, GradPtr grad_ptr)
 {
     constexpr int GB = VEC * G::kBytes;
     float p[VEC], v[VEC], sum[VEC];
-    load_state<VEC>(params + first, p);
-    load_state<VEC>(momentum + first, v);
+    load_state<VEC>(state_ptr(0) + first, p);
+    load_state<VEC>(state_ptr(1) + first, v);
     // -0.0f is the additive identity of IEEE addition (x + -0 == x for every x,
     // including x == -0), so a running sum started there equals the plain
     // left-to-right sum that starts at the first member.
@@ -221,8 +228,8 @@ __device__ __forceinline__ void update_vector(float *__restrict__ params, float 
             }
         }
     }
-    store_state<VEC>(params + first, p);
-    store_state<VEC>(momentum + first, v);
+    store_state<VEC>(state_ptr(0) + first, p);
+    store_state<VEC>(state_ptr(1) + first, v);
 }
 
 // ---------------------------------------------------------------------------
@@ -241,18 +248,19 @@ struct FlatArgs {
 // Grid-stride over vectors; the last < VEC elements are done one by one by the
 // first threads of block 0.
 template <typename G, int VEC, int DEPTH>
-__global__ void __launch_bounds__(kBlockThreads)
+__global__ void __launch_bounds__(kBlockThreads, kResidentBlocks)
 star_update_flat_kernel(const __grid_constant__ FlatArgs a)
 {
     const int64_t n_vec = a.n / VEC;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlockThreads;
     auto grad_ptr = [&](int slot) -> const void * { return a.grads[a.sched.member[slot]]; };
+    auto state_ptr = [&](int which) -> float * { return which == 0 ? a.params : a.momentum; };
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kBlockThreads + threadIdx.x; i < n_vec; i += stride)
-        update_vector<G, VEC, DEPTH>(a.params, a.momentum, i * VEC, a.sched, a.hyper, grad_ptr);
+        update_vector<G, VEC, DEPTH>(state_ptr, i * VEC, a.sched, a.hyper, grad_ptr);
     if constexpr (VEC > 1) {
         const int64_t tail = n_vec * VEC + threadIdx.x;
         if (blockIdx.x == 0 && threadIdx.x < VEC && tail < a.n)
-            update_vector<G, 1, DEPTH>(a.params, a.momentum, tail, a.sched, a.hyper, grad_ptr);
+            update_vector<G, 1, DEPTH>(state_ptr, tail, a.sched, a.hyper, grad_ptr);
     }
 }
 
@@ -281,34 +289,57 @@ struct MultiArgs {
     Hyper hyper;
 };
 
-template <typename G, int VEC, int DEPTH, int VEC_PER_THREAD>
-__global__ void __launch_bounds__(kBlockThreads)
+// Element-by-element path for the ragged end of a tensor and for tensors whose
+// buffers are not aligned for vector access.  Kept out of line: it is cold, and
+// inlining it next to the vector path costs registers there.
+template <typename G, int DEPTH>
+__device__ __noinline__ void update_elements(const TensorEntry &te, const unsigned long long *row,
+                                             int64_t first, int64_t end, int64_t step,
+                                             const FlatSchedule &s, const Hyper &h)
+{
+    auto grad_ptr = [&](int slot) -> const void * {
+        return reinterpret_cast<const void *>(__ldg(row + s.member[slot]));
+    };
+    auto state_ptr = [&](int which) -> float * { return which == 0 ? te.params : te.momentum; };
+    for (int64_t i = first; i < end; i += step)
+        update_vector<G, 1, DEPTH>(state_ptr, i, s, h, grad_ptr);
+}
+
+// One block per tile of kBlockThreads * VEC elements (grid-stride over tiles);
+// a thread owns one vector of its tile.
+template <typename G, int VEC, int DEPTH>
+__global__ void __launch_bounds__(kBlockThreads, kResidentBlocks)
 star_update_multi_kernel(const __grid_constant__ MultiArgs a)
 {
-    constexpr int64_t kTile = static_cast<int64_t>(kBlockThreads) * VEC * VEC_PER_THREAD;
+    constexpr int64_t kTile = static_cast<int64_t>(kBlockThreads) * VEC;
     for (int64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
         const int32_t t = __ldg(a.tile_tensor + tile);
-        const TensorEntry te = a.tensors[t];
+        const TensorEntry &te = a.tensors[t];
         const unsigned long long *row =
             reinterpret_cast<const unsigned long long *>(a.grads) + static_cast<int64_t>(t) * a.W;
-        auto grad_ptr = [&](int slot) -> const void * {
-            return reinterpret_cast<const void *>(__ldg(row + a.sched.member[slot]));
-        };
         const int64_t begin = (tile - te.first_tile) * kTile;
-        const int64_t end = min(te.size, begin + kTile);
+        const int64_t size = te.size;
         if (te.vector_ok) {
-            const int64_t vec_end = begin + (end - begin) / VEC * VEC;
-#pragma unroll 1
-            for (int64_t i = begin + static_cast<int64_t>(threadIdx.x) * VEC; i < vec_end;
-                 i += static_cast<int64_t>(kBlockThreads) * VEC)
-                update_vector<G, VEC, DEPTH>(te.params, te.momentum, i, a.sched, a.hyper, grad_ptr);
-            if (vec_end + threadIdx.x < end)         // fewer than VEC leftovers
-                update_vector<G, 1, DEPTH>(te.params, te.momentum, vec_end + threadIdx.x, a.sched,
-                                           a.hyper, grad_ptr);
+            const int64_t i = begin + static_cast<int64_t>(threadIdx.x) * VEC;
+            if (i + VEC <= size) {
+                auto grad_ptr = [&](int slot) -> const void * {
+                    return reinterpret_cast<const void *>(__ldg(row + a.sched.member[slot]));
+                };
+                // Re-read the bases from the (L1-resident) entry instead of
+                // keeping four registers live across the update.
+                auto state_ptr = [&](int which) -> float * {
+                    unsigned long long base;
+                    asm volatile("ld.global.nc.u64 %0, [%1];" : "=l"(base)
+                                 : "l"(which == 0 ? &te.params : &te.momentum));
+                    return reinterpret_cast<float *>(base);
+                };
+                update_vector<G, VEC, DEPTH>(state_ptr, i, a.sched, a.hyper, grad_ptr);
+            } else if (i < size) {                   // the tensor's last, partial vector
+                update_elements<G, DEPTH>(te, row, i, size, 1, a.sched, a.hyper);
+            }
         } else {
-#pragma unroll 1
-            for (int64_t i = begin + threadIdx.x; i < end; i += kBlockThreads)
-                update_vector<G, 1, DEPTH>(te.params, te.momentum, i, a.sched, a.hyper, grad_ptr);
+            const int64_t end = min(size, begin + kTile);
+            update_elements<G, DEPTH>(te, row, begin + threadIdx.x, end, kBlockThreads, a.sched, a.hyper);
         }
     }
 }
