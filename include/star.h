@@ -184,6 +184,47 @@ STAR_API star_status_t star_group_update_multi(const star_multi_plan_t *plan,
                                       int n_groups, float lr, float mu, float wd,
                                       void *cuda_stream);
 
+/* ---------------------------------------------------------------------------
+ * Tensor-list round for callers that cannot allocate device memory.
+ *
+ * The paper has no counterpart to this entry point; it exists for integration.
+ * Some callers of this library are not in a position to call cudaMalloc or to
+ * obtain a workspace from an allocator: a plug-in that runs inside another
+ * framework's step after that framework's pool has taken all free device
+ * memory, a hook on a latency-critical path where cudaMalloc's device-wide
+ * synchronization is not acceptable, or early start-up code that runs before
+ * any allocator exists.  For them the pointer table and tile map that
+ * star_multi_prepare would place in a caller workspace live in a fixed array of
+ * STAR_STATIC_SCRATCH_BYTES inside the library's device image (each GPU that
+ * loads the library holds that much until the process exits).
+ *
+ * The call does the work of star_multi_prepare followed by
+ * star_group_update_multi: arguments have the same meaning as there, and the
+ * results are identical.  It calls no cudaMalloc, cudaFree or other allocating
+ * routine.  Differences to know about:
+ *   - Size limit: a list whose table needs more than STAR_STATIC_SCRATCH_BYTES
+ *     (see star_multi_workspace_bytes) is rejected with
+ *     STAR_ERR_WORKSPACE_TOO_SMALL and nothing is launched.  1 MiB covers, for
+ *     example, 292 tensors / 355 M elements / 16 workers (about 0.75 MiB).
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous
+ *     call's table; each call rewrites the part it uses before its kernel
+ *     reads it, so nothing has to start out zeroed.  Calls on one stream are
+ *     ordered and safe.  Calls that can overlap on the GPU (different streams
+ *     without a dependency, or several host threads) race on the array: the
+ *     caller must serialize them.
+ *   - The table is rebuilt and copied (one cudaMemcpyAsync from pageable host
+ *     memory) on every call; callers that can provide a workspace should
+ *     prepare once and use star_group_update_multi.
+ * ------------------------------------------------------------------------- */
+#define STAR_STATIC_SCRATCH_BYTES (1u << 20)
+
+STAR_API star_status_t star_group_update_multi_noalloc(
+    int n_tensors, float *const *params, float *const *momentum, const void *const *grads,
+    const int64_t *sizes, int W, star_dtype_t grad_dtype, const int32_t *group_offsets,
+    const int32_t *group_members, int n_groups, float lr, float mu, float wd, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

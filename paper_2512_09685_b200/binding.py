@@ -80,6 +80,9 @@ def _load() -> ctypes.CDLL:
     lib.star_multi_prepare.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp,
                                        ctypes.c_size_t, c_vp, c_vp]
     lib.star_group_update_multi.argtypes = [c_vp, c_vp, c_vp, c_int, c_f, c_f, c_f, c_vp]
+    lib.star_group_update_multi_noalloc.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp, c_vp,
+                                                    c_int, c_f, c_f, c_f, c_vp]
+    lib.star_group_update_multi_noalloc.restype = c_int
     for name in ("star_schedule_validate", "star_schedule_static_x", "star_schedule_from_labels",
                  "star_schedule_dynamic_x", "star_group_update", "star_multi_workspace_bytes",
                  "star_multi_prepare", "star_group_update_multi"):
@@ -277,3 +280,49 @@ def star_group_update_multi(plan: star_multi_plan_t, group_offsets: Sequence[int
     K = len(group_offsets) - 1 if len(group_offsets) else 0
     _check(_lib.star_group_update_multi(ctypes.byref(plan), _i32(group_offsets), _i32(group_members),
                                         K, lr, mu, wd, _stream(stream)), "star_group_update_multi")
+
+
+STAR_STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def star_group_update_multi_noalloc(params: Sequence[torch.Tensor], momentum: Sequence[torch.Tensor],
+                                    grads: Sequence[Sequence[Optional[torch.Tensor]]],
+                                    group_offsets: Sequence[int], group_members: Sequence[int],
+                                    lr: float, mu: float, wd: float, stream=None) -> None:
+    """One round over a tensor list for callers that have no way to obtain a
+    device workspace (``grads[w][t]`` = worker w's gradient for tensor t).
+
+    The pointer table goes into a fixed array inside the library
+    (``STAR_STATIC_SCRATCH_BYTES``) that every call on the device shares; lists
+    whose table is larger are rejected with ``STAR_ERR_WORKSPACE_TOO_SMALL``.
+    Results equal :func:`star_multi_prepare` + :func:`star_group_update_multi`.
+    The caller must serialize calls that could overlap on the GPU, and should
+    make the first call on each device outside stream capture."""
+    T, W = len(params), len(grads)
+    if len(momentum) != T or any(len(g) != T for g in grads):
+        raise ValueError("params, momentum and every worker's gradient list need one entry per tensor")
+    sizes = [p.numel() for p in params]
+    if any(v.numel() != s for v, s in zip(momentum, sizes)):
+        raise ValueError("params and momentum differ in size")
+    P = (ctypes.c_void_p * max(T, 1))(*[_state(p, "params") if p.numel() else None for p in params])
+    V = (ctypes.c_void_p * max(T, 1))(*[_state(v, "momentum") if v.numel() else None for v in momentum])
+    G = (ctypes.c_void_p * max(T * W, 1))()
+    dt = None
+    for w in range(W):
+        for t in range(T):
+            g = grads[w][t]
+            if g is None or sizes[t] == 0:
+                continue
+            if not g.is_cuda or not g.is_contiguous() or g.numel() != sizes[t]:
+                raise ValueError("gradient [%d][%d] must be a contiguous CUDA tensor of %d elements"
+                                 % (w, t, sizes[t]))
+            d = _grad_dtype(g)
+            if dt is not None and d != dt:
+                raise TypeError("gradients differ in dtype")
+            dt = d
+            G[t * W + w] = g.data_ptr()
+    S = (ctypes.c_int64 * max(T, 1))(*sizes)
+    K = len(group_offsets) - 1 if len(group_offsets) else 0
+    _check(_lib.star_group_update_multi_noalloc(T, P, V, G, S, W, STAR_DTYPE_F32 if dt is None else dt,
+                                                _i32(group_offsets), _i32(group_members), K, lr, mu, wd,
+                                                _stream(stream)), "star_group_update_multi_noalloc")

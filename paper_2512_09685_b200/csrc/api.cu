@@ -359,3 +359,60 @@ extern "C" star_status_t star_group_update_multi(const star_multi_plan_t *plan,
     if (dt == STAR_DTYPE_F32) return launch_multi<GradF32, kVecF32>(args, stream);
     return STAR_ERR_INVALID_ARG;
 }
+
+// ---------------------------------------------------------------------------
+// Tensor-list round without any allocation: the table lives in a fixed array
+// of the library's own device image.
+// ---------------------------------------------------------------------------
+namespace {
+
+// In host code this name is only a handle for the runtime's symbol lookup, not
+// an address a kernel could use; the device address comes from
+// cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[STAR_STATIC_SCRATCH_BYTES];
+
+std::atomic<void *> g_static_scratch_address[kMaxDevices];
+
+// Device address of the array on the current device, looked up on first use.
+cudaError_t static_scratch_address(void **out)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    void *ptr = g_static_scratch_address[dev].load(std::memory_order_acquire);
+    if (!ptr) {
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        if (!ptr) return cudaErrorInvalidSymbol;
+        g_static_scratch_address[dev].store(ptr, std::memory_order_release);   // same value from any thread
+    }
+    *out = ptr;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" star_status_t star_group_update_multi_noalloc(
+    int n_tensors, float *const *params, float *const *momentum, const void *const *grads,
+    const int64_t *sizes, int W, star_dtype_t grad_dtype, const int32_t *group_offsets,
+    const int32_t *group_members, int n_groups, float lr, float mu, float wd, void *cuda_stream)
+{
+    // Reject a bad schedule before the shared table is touched.
+    star_status_t st = star_schedule_validate(group_offsets, group_members, n_groups, W);
+    if (st != STAR_OK) return st;
+    size_t need = 0;
+    st = star_multi_workspace_bytes(n_tensors, sizes, W, &need);
+    if (st != STAR_OK) return st;
+    if (need > STAR_STATIC_SCRATCH_BYTES) return STAR_ERR_WORKSPACE_TOO_SMALL;
+    void *scratch = nullptr;
+    const cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return cuda_failed(e);
+    // The copy into the array is ordered on cuda_stream after the previous
+    // call's kernel and before this call's kernel.
+    star_multi_plan_t plan;
+    st = star_multi_prepare(n_tensors, params, momentum, grads, sizes, W, grad_dtype, scratch,
+                            STAR_STATIC_SCRATCH_BYTES, cuda_stream, &plan);
+    if (st != STAR_OK) return st;
+    return star_group_update_multi(&plan, group_offsets, group_members, n_groups, lr, mu, wd, cuda_stream);
+}
