@@ -308,6 +308,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default=HEADLINE)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n", type=int, default=0,
+                    help="run a flat workload at this many elements instead of its full size "
+                         "(small cases for profiler captures; not a benchmark configuration)")
     ap.add_argument("--no-extra", action="store_true",
                     help="skip the other workloads, the CPU baseline and the end-to-end leg")
     args = ap.parse_args()
@@ -336,6 +339,8 @@ def main():
         dist = dist_mod
 
     w = WL.BY_NAME[args.workload]
+    if args.n > 0:
+        w = WL.scaled(w, args.n)
     peak, peak_kind = measured_peak()
     dw = DeviceWorkload(w, grad_sets=2 if w.n * w.W * w.grad_bytes < (4 << 30) else 1)
     sampler = ClockSampler(local_rank)
