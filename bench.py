@@ -230,6 +230,63 @@ def time_device(dw: DeviceWorkload, steps: int, warmup: int, dist, sampler=None)
     return seconds, per_launch, nbytes, launches
 
 
+def time_e2e(w, steps: int, warmup: int, dist):
+    """The same rounds through the host-buffer entry point: p, v and gradients
+    start in pinned host memory and p, v end there; every copy is inside the
+    timed region and each step ends with the stream synchronized (the result
+    is read on the host).  Returns (seconds [max over ranks], bytes, h2d, d2h
+    per step, launches)."""
+    import torch
+    from paper_2512_09685_b200 import binding as B
+    from paper_2512_09685_b200 import workloads as WL
+    n = w.n
+    flat = WL.scaled(w, n)                      # tensor lists are streamed as one flat buffer
+    p = WL.make_params(flat, "cpu")[0].pin_memory()
+    v = WL.make_momentum(flat, "cpu")[0].pin_memory()
+    one = torch.empty(n, dtype=w.torch_grad_dtype())
+    WL.fill_grads(flat, 0, 0, [one])
+    grads = []
+    for wk in range(w.W):                       # values do not affect the timing: one draw, W pinned copies
+        g = torch.empty(n, dtype=w.torch_grad_dtype()).pin_memory()
+        g.copy_(one)
+        grads.append(g)
+    chunk = 4 * 1024 * 1024
+    ws = torch.empty(B.star_host_workspace_bytes(w.W, w.torch_grad_dtype(), chunk), dtype=torch.uint8,
+                     device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        off, mem = B.encode(w.decision(i))
+        B.star_group_update_host(p, v, grads, off, mem, w.lr, w.mu, w.wd, ws)
+        stream.synchronize()
+        return off[-1]
+
+    for i in range(warmup):
+        step(i)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = B.star_launch_count()
+    scheduled = 0
+    e0.record()
+    for i in range(steps):
+        scheduled += step(warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    seconds = e0.elapsed_time(e1) / 1e3
+    if dist is not None:
+        t = torch.tensor([seconds], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        seconds = float(t.item())
+    nbytes = n * (scheduled * w.grad_bytes + 16 * steps)
+    h2d = n * (scheduled * w.grad_bytes + 8 * steps) // steps
+    d2h = n * 8
+    return seconds, nbytes, h2d, d2h, B.star_launch_count() - launches0
+
+
 # ---------------------------------------------------------------------------
 # CPU oracle timing
 # ---------------------------------------------------------------------------
@@ -339,8 +396,10 @@ def main():
     ap.add_argument("--n", type=int, default=0,
                     help="run a flat workload at this many elements instead of its full size "
                          "(small cases for profiler captures; not a benchmark configuration)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-extra", action="store_true",
-                    help="skip the other workloads, the CPU baseline and the end-to-end leg")
+                    help="device-timed headline only: skip the end-to-end leg, the other workloads "
+                         "and the CPU baseline")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -399,9 +458,18 @@ def main():
                      "kernel_ms_min": min(per_launch)},
     }
 
+    del dw
+    torch.cuda.empty_cache()
+    if not args.no_e2e and not args.no_extra:
+        e2e_steps = max(3, min(args.steps, 20))
+        esec, ebytes, h2d, d2h, elaunch = time_e2e(w, e2e_steps, 3, dist)
+        out["e2e"] = {"value": ebytes / esec / 1e9 * world, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": esec / e2e_steps * 1e3,
+                      "gpu_launches": elaunch,
+                      "how": "star_group_update_host on pinned host tensors, 4 Mi-element chunks, "
+                             "stream synchronized every step"}
+
     if not args.no_extra and rank == 0 and world == 1:
-        del dw
-        torch.cuda.empty_cache()
         others = {}
         for other in WL.WORKLOADS:
             if other.name == w.name:

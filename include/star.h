@@ -185,6 +185,44 @@ STAR_API star_status_t star_group_update_multi(const star_multi_plan_t *plan,
                                       void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
+ * Fused grouped update with the state and the gradients in HOST memory (the
+ * paper's parameter server keeps its parameter and gradient copies in host
+ * memory, Section II).  Same operation and results as star_group_update; the
+ * data is streamed through the GPU in chunks: copy a chunk of p, v and of every
+ * scheduled worker's gradient to the device, run the fused kernel on it, copy
+ * p and v back, with the copies of neighbouring chunks overlapping (host to
+ * device on cuda_stream, device to host on an internal stream).
+ *   h_params, h_momentum : host, fp32, n elements, updated in place
+ *   h_grads              : host array of W host pointers (unscheduled: may be NULL)
+ *   d_workspace          : device, 256-byte aligned staging memory provided by
+ *                          the caller; star_host_workspace_bytes() gives the
+ *                          size for a chosen chunk length
+ * Host buffers should be page-locked (cudaHostAlloc / cudaHostRegister):
+ * pageable memory works but its copies do not overlap.  The call enqueues all
+ * work and returns; results are in the host buffers once cuda_stream has been
+ * synchronized.  The first call on a device creates one internal stream and a
+ * few events (no device memory).  Calls on the same device are serialized
+ * against each other at enqueue time by the library; they must not share a
+ * workspace unless they are ordered on one stream.
+ * ------------------------------------------------------------------------- */
+
+/* Workspace bytes for chunks of chunk_elements elements (a multiple of 2048, at
+ * least 2048) when at most max_scheduled workers are scheduled in a round. */
+STAR_API star_status_t star_host_workspace_bytes(int max_scheduled, star_dtype_t grad_dtype,
+                                                 int64_t chunk_elements, size_t *bytes_out);
+
+/* The chunk length is the largest multiple of 2048 that fits workspace_bytes for
+ * the number of workers this schedule uses; STAR_ERR_WORKSPACE_TOO_SMALL if
+ * that is below 2048.  One kernel launch per chunk. */
+STAR_API star_status_t star_group_update_host(float *h_params, float *h_momentum,
+                                              const void *const *h_grads, int W,
+                                              star_dtype_t grad_dtype, int64_t n,
+                                              const int32_t *group_offsets,
+                                              const int32_t *group_members, int n_groups, float lr,
+                                              float mu, float wd, void *d_workspace,
+                                              size_t workspace_bytes, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * Tensor-list round for callers that cannot allocate device memory.
  *
  * The paper has no counterpart to this entry point; it exists for integration.

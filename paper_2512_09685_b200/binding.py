@@ -80,6 +80,11 @@ def _load() -> ctypes.CDLL:
     lib.star_multi_prepare.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp,
                                        ctypes.c_size_t, c_vp, c_vp]
     lib.star_group_update_multi.argtypes = [c_vp, c_vp, c_vp, c_int, c_f, c_f, c_f, c_vp]
+    lib.star_host_workspace_bytes.argtypes = [c_int, c_int, c_i64, c_vp]
+    lib.star_host_workspace_bytes.restype = c_int
+    lib.star_group_update_host.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
+                                           c_f, c_f, c_f, c_vp, ctypes.c_size_t, c_vp]
+    lib.star_group_update_host.restype = c_int
     lib.star_group_update_multi_noalloc.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp, c_vp,
                                                     c_int, c_f, c_f, c_f, c_vp]
     lib.star_group_update_multi_noalloc.restype = c_int
@@ -280,6 +285,49 @@ def star_group_update_multi(plan: star_multi_plan_t, group_offsets: Sequence[int
     K = len(group_offsets) - 1 if len(group_offsets) else 0
     _check(_lib.star_group_update_multi(ctypes.byref(plan), _i32(group_offsets), _i32(group_members),
                                         K, lr, mu, wd, _stream(stream)), "star_group_update_multi")
+
+
+def star_host_workspace_bytes(max_scheduled: int, grad_dtype: torch.dtype, chunk_elements: int) -> int:
+    out = ctypes.c_size_t(0)
+    dt = STAR_DTYPE_BF16 if grad_dtype == torch.bfloat16 else STAR_DTYPE_F32
+    _check(_lib.star_host_workspace_bytes(max_scheduled, dt, chunk_elements, ctypes.byref(out)),
+           "star_host_workspace_bytes")
+    return out.value
+
+
+def star_group_update_host(params: torch.Tensor, momentum: torch.Tensor,
+                           grads: Sequence[Optional[torch.Tensor]], group_offsets: Sequence[int],
+                           group_members: Sequence[int], lr: float, mu: float, wd: float,
+                           workspace: torch.Tensor, stream=None) -> None:
+    """Fused grouped update of HOST tensors (ideally pinned), streamed through the
+    device workspace in chunks.  Results are in ``params`` / ``momentum`` once the
+    stream has been synchronized."""
+    n = params.numel()
+    for t, what in ((params, "params"), (momentum, "momentum")):
+        if t.dtype != torch.float32 or t.is_cuda or not t.is_contiguous():
+            raise TypeError("%s must be a contiguous float32 host tensor" % what)
+    if momentum.numel() != n:
+        raise ValueError("params and momentum differ in size")
+    W = len(grads)
+    ptrs = (ctypes.c_void_p * max(W, 1))()
+    dt = None
+    for w, g in enumerate(grads):
+        if g is None:
+            continue
+        if g.is_cuda or not g.is_contiguous() or g.numel() != n:
+            raise ValueError("gradient %d must be a contiguous host tensor of %d elements" % (w, n))
+        d = _grad_dtype(g)
+        if dt is not None and d != dt:
+            raise TypeError("gradients differ in dtype")
+        dt = d
+        ptrs[w] = g.data_ptr()
+    if workspace.dtype != torch.uint8 or not workspace.is_cuda or not workspace.is_contiguous():
+        raise TypeError("workspace must be a contiguous uint8 CUDA tensor")
+    K = len(group_offsets) - 1 if len(group_offsets) else 0
+    _check(_lib.star_group_update_host(params.data_ptr(), momentum.data_ptr(), ptrs, W,
+                                       STAR_DTYPE_F32 if dt is None else dt, n, _i32(group_offsets),
+                                       _i32(group_members), K, lr, mu, wd, workspace.data_ptr(),
+                                       workspace.numel(), _stream(stream)), "star_group_update_host")
 
 
 STAR_STATIC_SCRATCH_BYTES = 1 << 20

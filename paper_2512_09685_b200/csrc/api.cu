@@ -2,6 +2,7 @@
 #include <atomic>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include <cuda_runtime.h>
@@ -358,6 +359,174 @@ extern "C" star_status_t star_group_update_multi(const star_multi_plan_t *plan,
     if (dt == STAR_DTYPE_BF16) return launch_multi<GradBF16, kVecBF16>(args, stream);
     if (dt == STAR_DTYPE_F32) return launch_multi<GradF32, kVecF32>(args, stream);
     return STAR_ERR_INVALID_ARG;
+}
+
+// ---------------------------------------------------------------------------
+// Host-resident state and gradients: chunked, double-buffered streaming.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t kHostChunkQuantum = 2048;
+
+struct HostPipeline {            // per device, created on first use, never destroyed
+    cudaStream_t copy_back = nullptr;
+    cudaEvent_t kernel_done[2] = {nullptr, nullptr};
+    cudaEvent_t copied_back[2] = {nullptr, nullptr};
+    bool ready = false;
+};
+
+std::mutex g_host_mutex[kMaxDevices];
+HostPipeline g_host_pipeline[kMaxDevices];
+
+cudaError_t host_pipeline(int dev, HostPipeline **out)
+{
+    HostPipeline &hp = g_host_pipeline[dev];
+    if (!hp.ready) {
+        cudaError_t e = cudaStreamCreateWithFlags(&hp.copy_back, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return e;
+        for (int i = 0; i < 2; ++i) {
+            e = cudaEventCreateWithFlags(&hp.kernel_done[i], cudaEventDisableTiming);
+            if (e != cudaSuccess) return e;
+            e = cudaEventCreateWithFlags(&hp.copied_back[i], cudaEventDisableTiming);
+            if (e != cudaSuccess) return e;
+        }
+        hp.ready = true;
+    }
+    *out = &hp;
+    return cudaSuccess;
+}
+
+// Bytes of one staging set (p, v and `scheduled` gradient chunks), each
+// sub-buffer rounded up to the workspace alignment.
+size_t host_set_bytes(int scheduled, size_t gsize, int64_t chunk)
+{
+    const size_t state = round_up(static_cast<size_t>(chunk) * 4, kWorkspaceAlign);
+    const size_t grad = round_up(static_cast<size_t>(chunk) * gsize, kWorkspaceAlign);
+    return 2 * state + static_cast<size_t>(scheduled) * grad;
+}
+
+}  // namespace
+
+extern "C" star_status_t star_host_workspace_bytes(int max_scheduled, star_dtype_t grad_dtype,
+                                                   int64_t chunk_elements, size_t *bytes_out)
+{
+    if (!bytes_out) return STAR_ERR_NULL_POINTER;
+    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (max_scheduled < 0 || chunk_elements < kHostChunkQuantum || chunk_elements % kHostChunkQuantum != 0)
+        return STAR_ERR_INVALID_ARG;
+    if (max_scheduled > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    *bytes_out = 2 * host_set_bytes(max_scheduled, grad_dtype == STAR_DTYPE_BF16 ? 2 : 4, chunk_elements);
+    return STAR_OK;
+}
+
+extern "C" star_status_t star_group_update_host(float *h_params, float *h_momentum,
+                                                const void *const *h_grads, int W,
+                                                star_dtype_t grad_dtype, int64_t n,
+                                                const int32_t *group_offsets,
+                                                const int32_t *group_members, int n_groups, float lr,
+                                                float mu, float wd, void *d_workspace,
+                                                size_t workspace_bytes, void *cuda_stream)
+{
+    if (n < 0 || W < 0) return STAR_ERR_INVALID_ARG;
+    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    FlatArgs args;
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, lr, &args.sched);
+    if (st != STAR_OK) return st;
+    if (n == 0 || n_groups == 0) return STAR_OK;
+    if (!h_params || !h_momentum || !h_grads || !d_workspace) return STAR_ERR_NULL_POINTER;
+    if (!aligned(d_workspace, kWorkspaceAlign)) return STAR_ERR_INVALID_ARG;
+
+    const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const int scheduled = args.sched.n_slots;
+    const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
+    if (!aligned(h_params, 4) || !aligned(h_momentum, 4)) return STAR_ERR_INVALID_ARG;
+    if (overlaps(h_params, state_bytes, h_momentum, state_bytes)) return STAR_ERR_INVALID_ARG;
+    for (int j = 0; j < scheduled; ++j) {
+        const void *g = h_grads[args.sched.member[j]];
+        if (!g) return STAR_ERR_NULL_POINTER;
+        if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
+        if (overlaps(g, grad_bytes, h_params, state_bytes) || overlaps(g, grad_bytes, h_momentum, state_bytes))
+            return STAR_ERR_INVALID_ARG;
+    }
+    // Largest chunk (multiple of the quantum) whose two staging sets fit.
+    int64_t chunk = static_cast<int64_t>(workspace_bytes / (2 * (8 + static_cast<size_t>(scheduled) * gsize)));
+    chunk = chunk / kHostChunkQuantum * kHostChunkQuantum;
+    while (chunk >= kHostChunkQuantum && 2 * host_set_bytes(scheduled, gsize, chunk) > workspace_bytes)
+        chunk -= kHostChunkQuantum;
+    if (chunk < kHostChunkQuantum) return STAR_ERR_WORKSPACE_TOO_SMALL;
+    const int64_t needed = (n + kHostChunkQuantum - 1) / kHostChunkQuantum * kHostChunkQuantum;
+    if (chunk > needed) chunk = needed;
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_failed(e);
+    if (dev < 0 || dev >= kMaxDevices) return cuda_failed(cudaErrorInvalidDevice);
+    std::lock_guard<std::mutex> lock(g_host_mutex[dev]);
+    HostPipeline *hp = nullptr;
+    e = host_pipeline(dev, &hp);
+    if (e != cudaSuccess) return cuda_failed(e);
+
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t set_bytes = host_set_bytes(scheduled, gsize, chunk);
+    const size_t state_stride = round_up(static_cast<size_t>(chunk) * 4, kWorkspaceAlign);
+    const size_t grad_stride = round_up(static_cast<size_t>(chunk) * gsize, kWorkspaceAlign);
+    char *const base = static_cast<char *>(d_workspace);
+    args.hyper = Hyper{mu, wd};
+
+    // The staging sets may still be in use by an earlier call's copy-back
+    // (another stream): order this call's first writes after it.
+    for (int b = 0; b < 2; ++b) {
+        e = cudaStreamWaitEvent(stream, hp->copied_back[b], 0);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
+    int64_t index = 0;
+    for (int64_t first = 0; first < n; first += chunk, ++index) {
+        const int b = static_cast<int>(index & 1);
+        const int64_t count = n - first < chunk ? n - first : chunk;
+        char *set = base + static_cast<size_t>(b) * set_bytes;
+        float *d_p = reinterpret_cast<float *>(set);
+        float *d_v = reinterpret_cast<float *>(set + state_stride);
+        if (index >= 2) {                       // set b was last used by chunk index - 2
+            e = cudaStreamWaitEvent(stream, hp->copied_back[b], 0);
+            if (e != cudaSuccess) return cuda_failed(e);
+        }
+        e = cudaMemcpyAsync(d_p, h_params + first, static_cast<size_t>(count) * 4, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = cudaMemcpyAsync(d_v, h_momentum + first, static_cast<size_t>(count) * 4, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return cuda_failed(e);
+        std::memset(args.grads, 0, sizeof args.grads);
+        for (int j = 0; j < scheduled; ++j) {
+            const int w = args.sched.member[j];
+            char *d_g = set + 2 * state_stride + static_cast<size_t>(j) * grad_stride;
+            const char *h_g = static_cast<const char *>(h_grads[w]) + static_cast<size_t>(first) * gsize;
+            e = cudaMemcpyAsync(d_g, h_g, static_cast<size_t>(count) * gsize, cudaMemcpyHostToDevice, stream);
+            if (e != cudaSuccess) return cuda_failed(e);
+            args.grads[w] = d_g;
+        }
+        args.params = d_p;
+        args.momentum = d_v;
+        args.n = count;
+        const star_status_t ls = grad_dtype == STAR_DTYPE_BF16 ? launch_flat<GradBF16, kVecBF16>(args, stream)
+                                                               : launch_flat<GradF32, kVecF32>(args, stream);
+        if (ls != STAR_OK) return ls;
+        e = cudaEventRecord(hp->kernel_done[b], stream);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = cudaStreamWaitEvent(hp->copy_back, hp->kernel_done[b], 0);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = cudaMemcpyAsync(h_params + first, d_p, static_cast<size_t>(count) * 4, cudaMemcpyDeviceToHost, hp->copy_back);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = cudaMemcpyAsync(h_momentum + first, d_v, static_cast<size_t>(count) * 4, cudaMemcpyDeviceToHost, hp->copy_back);
+        if (e != cudaSuccess) return cuda_failed(e);
+        e = cudaEventRecord(hp->copied_back[b], hp->copy_back);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
+    // Later work on the caller's stream (and its synchronize) sees the results.
+    for (int b = 0; b < 2; ++b) {
+        e = cudaStreamWaitEvent(stream, hp->copied_back[b], 0);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
+    return STAR_OK;
 }
 
 // ---------------------------------------------------------------------------
