@@ -193,6 +193,16 @@ class DeviceWorkload:
             v.zero_()
 
 
+def max_over_ranks(seconds: float, dist, device) -> float:
+    """The slowest rank's time: what a multi-rank measurement reports."""
+    if dist is None:
+        return seconds
+    import torch
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def time_device(dw: DeviceWorkload, steps: int, warmup: int, dist, sampler=None):
     """Returns (seconds for `steps` rounds [max over ranks], per-launch ms list,
     algorithmic bytes of those rounds on this rank, launches)."""
@@ -222,11 +232,7 @@ def time_device(dw: DeviceWorkload, steps: int, warmup: int, dist, sampler=None)
     total_ms = events[0].elapsed_time(events[steps])
     per_launch = [events[i].elapsed_time(events[i + 1]) for i in range(steps)]
     nbytes = dw.w.n * (scheduled * dw.w.grad_bytes + 16 * steps)
-    seconds = total_ms / 1e3
-    if dist is not None:
-        t = torch.tensor([seconds], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        seconds = float(t.item())
+    seconds = max_over_ranks(total_ms / 1e3, dist, "cuda")
     return seconds, per_launch, nbytes, launches
 
 
@@ -276,11 +282,7 @@ def time_e2e(w, steps: int, warmup: int, dist):
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
-    seconds = e0.elapsed_time(e1) / 1e3
-    if dist is not None:
-        t = torch.tensor([seconds], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        seconds = float(t.item())
+    seconds = max_over_ranks(e0.elapsed_time(e1) / 1e3, dist, "cuda")
     nbytes = n * (scheduled * w.grad_bytes + 16 * steps)
     h2d = n * (scheduled * w.grad_bytes + 8 * steps) // steps
     d2h = n * 8

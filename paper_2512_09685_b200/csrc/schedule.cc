@@ -147,3 +147,22 @@ extern "C" star_status_t star_schedule_dynamic_x(const double *iter_time, const 
     pack(groups, offsets_out, members_out, n_groups_out);
     return STAR_OK;
 }
+
+extern "C" star_status_t star_shard_range(int64_t n, int world, int rank, int64_t align,
+                                          int64_t *first_out, int64_t *count_out)
+{
+    if (!first_out || !count_out) return STAR_ERR_NULL_POINTER;
+    if (n < 0 || world < 1 || rank < 0 || rank >= world || align < 1) return STAR_ERR_INVALID_ARG;
+    // Split the ceil(n / align) blocks of `align` elements as evenly as possible;
+    // the last block may be partial.
+    const int64_t blocks = (n + align - 1) / align;
+    const int64_t base = blocks / world, extra = blocks % world;
+    const int64_t first_block = base * rank + (rank < extra ? rank : extra);
+    const int64_t n_blocks = base + (rank < extra ? 1 : 0);
+    int64_t first = first_block * align, last = (first_block + n_blocks) * align;
+    if (first > n) first = n;
+    if (last > n) last = n;
+    *first_out = first;
+    *count_out = last - first;
+    return STAR_OK;
+}
