@@ -213,15 +213,15 @@ def time_device(dw: DeviceWorkload, steps: int, warmup: int, dist, sampler=None)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    events = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    begin, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = B.star_launch_count()
     scheduled = 0
     if sampler is not None:
         sampler.__enter__()
-    events[0].record()
+    begin.record()
     for i in range(steps):
         scheduled += dw.step()
-        events[i + 1].record()
+    end.record()
     torch.cuda.synchronize()
     if sampler is not None:
         sampler.__exit__(None, None, None)
@@ -229,8 +229,18 @@ def time_device(dw: DeviceWorkload, steps: int, warmup: int, dist, sampler=None)
         dist.barrier()
     torch.cuda.synchronize()
     launches = B.star_launch_count() - launches0
-    total_ms = events[0].elapsed_time(events[steps])
-    per_launch = [events[i].elapsed_time(events[i + 1]) for i in range(steps)]
+    total_ms = begin.elapsed_time(end)
+    # Per-launch durations from a short extra pass with an event after every
+    # launch (the events themselves cost time, so they stay out of the timed
+    # region above; the pass only shows the spread).
+    probe = min(steps, 200)
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(probe + 1)]
+    events[0].record()
+    for i in range(probe):
+        dw.step()
+        events[i + 1].record()
+    torch.cuda.synchronize()
+    per_launch = [events[i].elapsed_time(events[i + 1]) for i in range(probe)]
     nbytes = dw.w.n * (scheduled * dw.w.grad_bytes + 16 * steps)
     seconds = max_over_ranks(total_ms / 1e3, dist, "cuda")
     return seconds, per_launch, nbytes, launches
@@ -436,7 +446,9 @@ def main():
     seconds, per_launch, nbytes, launches = time_device(dw, args.steps, args.warmup, dist, sampler)
     gbs_rank = nbytes / seconds / 1e9
     value = gbs_rank * world
-    kernel_ms = statistics.mean(per_launch)
+    # one launch per step and nothing else on the stream: the kernel's mean
+    # launch duration over the timed region is the region's time / launches
+    kernel_ms = seconds / launches * 1e3
     achieved = (nbytes / args.steps) / (kernel_ms / 1e3) / 1e9
 
     out = {
@@ -456,8 +468,9 @@ def main():
                      "frac": achieved / peak,
                      "traffic": ncu_traffic(w.name) if args.n <= 0 else None, "peak_kind": "of " + peak_kind,
                      "kernel": "star_update_multi_kernel" if w.multi_tensor else "star_update_flat_kernel",
-                     "kernel_ms_mean": kernel_ms, "kernel_ms_median": statistics.median(per_launch),
-                     "kernel_ms_min": min(per_launch)},
+                     "kernel_ms_mean": kernel_ms,
+                     "per_launch_probe_ms": {"median": statistics.median(per_launch), "min": min(per_launch),
+                                             "launches": len(per_launch)}},
     }
 
     del dw
