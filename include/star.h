@@ -143,6 +143,27 @@ STAR_API star_status_t star_group_update(float *params, float *momentum, const v
                                 const int32_t *group_offsets, const int32_t *group_members,
                                 int n_groups, float lr, float mu, float wd, void *cuda_stream);
 
+/* The same round with one learning rate per group and optional parameter
+ * snapshots.
+ *   lrs        : host, n_groups learning rates.  Section IV-C1 ("Scaling learning
+ *                rate after switching") sets the rate of an update built from y
+ *                gradient reports to (y / N) x the SSGD rate; the caller computes
+ *                the rates, the kernel applies lrs[k] in group k's update.
+ *   snapshots  : NULL, or host array of n_groups device pointers (fp32, n
+ *                elements each, entries may be NULL).  snapshots[k] receives the
+ *                parameters as they stand right after group k's update -- the
+ *                copy the server sends back to that group's workers (Section II)
+ *                -- written in the same pass (4 n more bytes of traffic each).
+ *                Snapshot buffers must not overlap each other or any other
+ *                buffer of the call.
+ * Everything else as star_group_update.  One kernel launch. */
+STAR_API star_status_t star_group_update_ex(float *params, float *momentum, const void *const *grads,
+                                            int W, star_dtype_t grad_dtype, int64_t n,
+                                            const int32_t *group_offsets,
+                                            const int32_t *group_members, int n_groups,
+                                            const float *lrs, float mu, float wd,
+                                            float *const *snapshots, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------
  * Fused grouped update of a LIST of tensors (per-layer parameters) in one
  * launch.  The pointer table and tile map live in a caller-provided device

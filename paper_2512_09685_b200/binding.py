@@ -80,6 +80,9 @@ def _load() -> ctypes.CDLL:
     lib.star_multi_prepare.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp,
                                        ctypes.c_size_t, c_vp, c_vp]
     lib.star_group_update_multi.argtypes = [c_vp, c_vp, c_vp, c_int, c_f, c_f, c_f, c_vp]
+    lib.star_group_update_ex.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
+                                         c_vp, c_f, c_f, c_vp, c_vp]
+    lib.star_group_update_ex.restype = c_int
     lib.star_shard_range.argtypes = [c_i64, c_int, c_int, c_i64, c_vp, c_vp]
     lib.star_shard_range.restype = c_int
     lib.star_host_workspace_bytes.argtypes = [c_int, c_int, c_i64, c_vp]
@@ -240,6 +243,50 @@ def star_group_update(params: torch.Tensor, momentum: torch.Tensor,
     _check(_lib.star_group_update(p, v, ptrs, W, STAR_DTYPE_F32 if dt is None else dt, n,
                                   _i32(group_offsets), _i32(group_members), K, lr, mu, wd,
                                   _stream(stream)), "star_group_update")
+
+
+def star_group_update_ex(params: torch.Tensor, momentum: torch.Tensor,
+                         grads: Sequence[Optional[torch.Tensor]], group_offsets: Sequence[int],
+                         group_members: Sequence[int], lrs: Sequence[float], mu: float, wd: float,
+                         snapshots: Optional[Sequence[Optional[torch.Tensor]]] = None,
+                         stream=None) -> None:
+    """The round with one learning rate per group; ``snapshots[k]`` (fp32 CUDA
+    tensor or None) receives the parameters right after group k's update."""
+    n = params.numel()
+    p, v = _state(params, "params"), _state(momentum, "momentum")
+    if momentum.numel() != n:
+        raise ValueError("params and momentum differ in size")
+    W = len(grads)
+    ptrs = (ctypes.c_void_p * max(W, 1))()
+    dt = None
+    for w, g in enumerate(grads):
+        if g is None:
+            continue
+        if not g.is_cuda or not g.is_contiguous() or g.numel() != n:
+            raise ValueError("gradient %d must be a contiguous CUDA tensor of %d elements" % (w, n))
+        d = _grad_dtype(g)
+        if dt is not None and d != dt:
+            raise TypeError("gradients differ in dtype")
+        dt = d
+        ptrs[w] = g.data_ptr()
+    K = len(group_offsets) - 1 if len(group_offsets) else 0
+    if len(lrs) != K:
+        raise ValueError("need one learning rate per group")
+    lr_arr = (ctypes.c_float * max(K, 1))(*lrs)
+    snap_arr = None
+    if snapshots is not None:
+        if len(snapshots) != K:
+            raise ValueError("snapshots needs one entry (tensor or None) per group")
+        snap_arr = (ctypes.c_void_p * max(K, 1))()
+        for k, s in enumerate(snapshots):
+            if s is None:
+                continue
+            if s.numel() != n:
+                raise ValueError("snapshot %d differs in size" % k)
+            snap_arr[k] = _state(s, "snapshot")
+    _check(_lib.star_group_update_ex(p, v, ptrs, W, STAR_DTYPE_F32 if dt is None else dt, n,
+                                     _i32(group_offsets), _i32(group_members), K, lr_arr, mu, wd,
+                                     snap_arr, _stream(stream)), "star_group_update_ex")
 
 
 def star_multi_workspace_bytes(sizes: Sequence[int], W: int) -> int:

@@ -79,7 +79,7 @@ int choose_grid(int64_t work, int resident)
 // Schedule: validate, then flatten into the kernel's slot list.
 // ---------------------------------------------------------------------------
 star_status_t flatten_schedule(const int32_t *group_offsets, const int32_t *group_members, int n_groups,
-                               int W, float lr, FlatSchedule *out)
+                               int W, float lr, FlatSchedule *out, const float *lrs = nullptr)
 {
     const star_status_t st = star_schedule_validate(group_offsets, group_members, n_groups, W);
     if (st != STAR_OK) return st;
@@ -89,7 +89,7 @@ star_status_t flatten_schedule(const int32_t *group_offsets, const int32_t *grou
         const int first = group_offsets[k], last = group_offsets[k + 1];
         for (int j = first; j < last; ++j) out->member[j] = static_cast<uint8_t>(group_members[j]);
         out->group_size[last - 1] = static_cast<uint8_t>(last - first);
-        out->neg_lr[last - 1] = -lr;
+        out->neg_lr[last - 1] = lrs ? -lrs[k] : -lr;
     }
     return STAR_OK;
 }
@@ -187,6 +187,95 @@ extern "C" star_status_t star_group_update(float *params, float *momentum, const
     if (grad_dtype == STAR_DTYPE_BF16)
         return vector_ok ? launch_flat<GradBF16, kVecBF16>(args, stream) : launch_flat<GradBF16, 1>(args, stream);
     return vector_ok ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
+}
+
+// Per-group learning rates and parameter snapshots.
+namespace {
+
+template <typename G, int VEC>
+star_status_t launch_flat_snapshot(const SnapshotArgs &args, cudaStream_t stream)
+{
+    static Geometry cache[kMaxDevices];
+    constexpr int depth = VEC == 1 ? kDepthScalar : kDepthVector;
+    auto kernel = star_update_flat_snapshot_kernel<G, VEC, depth>;
+    int blocks = 0;
+    cudaError_t e = resident_blocks(kernel, cache, &blocks);
+    if (e != cudaSuccess) return cuda_failed(e);
+    const int64_t work = (args.flat.n / VEC + kBlockThreads - 1) / kBlockThreads;
+    const int grid = choose_grid(work, blocks);
+    kernel<<<grid, kBlockThreads, 0, stream>>>(args);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return STAR_OK;
+}
+
+}  // namespace
+
+extern "C" star_status_t star_group_update_ex(float *params, float *momentum, const void *const *grads,
+                                              int W, star_dtype_t grad_dtype, int64_t n,
+                                              const int32_t *group_offsets, const int32_t *group_members,
+                                              int n_groups, const float *lrs, float mu, float wd,
+                                              float *const *snapshots, void *cuda_stream)
+{
+    if (n < 0 || W < 0) return STAR_ERR_INVALID_ARG;
+    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
+    SnapshotArgs sargs;
+    FlatArgs &args = sargs.flat;
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, 0.0f, &args.sched, lrs);
+    if (st != STAR_OK) return st;
+    if (n == 0 || n_groups == 0) return STAR_OK;
+    if (!params || !momentum || !grads) return STAR_ERR_NULL_POINTER;
+
+    const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
+    if (!aligned(params, 4) || !aligned(momentum, 4)) return STAR_ERR_INVALID_ARG;
+    if (overlaps(params, state_bytes, momentum, state_bytes)) return STAR_ERR_INVALID_ARG;
+    bool vector_ok = aligned(params, kVectorBytes) && aligned(momentum, kVectorBytes);
+    std::memset(args.grads, 0, sizeof args.grads);
+    for (int j = 0; j < args.sched.n_slots; ++j) {
+        const int w = args.sched.member[j];
+        const void *g = grads[w];
+        if (!g) return STAR_ERR_NULL_POINTER;
+        if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
+        if (overlaps(g, grad_bytes, params, state_bytes) || overlaps(g, grad_bytes, momentum, state_bytes))
+            return STAR_ERR_INVALID_ARG;
+        vector_ok = vector_ok && aligned(g, kVectorBytes);
+        args.grads[w] = g;
+    }
+    std::memset(sargs.snapshots, 0, sizeof sargs.snapshots);
+    bool any_snapshot = false;
+    for (int k = 0; snapshots && k < n_groups; ++k) {
+        float *snap = snapshots[k];
+        if (!snap) continue;
+        if (!aligned(snap, 4)) return STAR_ERR_INVALID_ARG;
+        if (overlaps(snap, state_bytes, params, state_bytes) || overlaps(snap, state_bytes, momentum, state_bytes))
+            return STAR_ERR_INVALID_ARG;
+        for (int j = 0; j < args.sched.n_slots; ++j)
+            if (overlaps(snap, state_bytes, args.grads[args.sched.member[j]], grad_bytes)) return STAR_ERR_INVALID_ARG;
+        for (int l = 0; l < k; ++l)
+            if (snapshots[l] && overlaps(snap, state_bytes, snapshots[l], state_bytes)) return STAR_ERR_INVALID_ARG;
+        vector_ok = vector_ok && aligned(snap, kVectorBytes);
+        sargs.snapshots[group_offsets[k + 1] - 1] = snap;
+        any_snapshot = true;
+    }
+    args.params = params;
+    args.momentum = momentum;
+    args.n = n;
+    args.hyper = Hyper{mu, wd};
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (!any_snapshot) {                       // per-group rates only: the plain kernel does it
+        if (grad_dtype == STAR_DTYPE_BF16)
+            return vector_ok ? launch_flat<GradBF16, kVecBF16>(args, stream) : launch_flat<GradBF16, 1>(args, stream);
+        return vector_ok ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
+    }
+    if (grad_dtype == STAR_DTYPE_BF16)
+        return vector_ok ? launch_flat_snapshot<GradBF16, kVecBF16>(sargs, stream)
+                         : launch_flat_snapshot<GradBF16, 1>(sargs, stream);
+    return vector_ok ? launch_flat_snapshot<GradF32, kVecF32>(sargs, stream)
+                     : launch_flat_snapshot<GradF32, 1>(sargs, stream);
 }
 
 // ---------------------------------------------------------------------------

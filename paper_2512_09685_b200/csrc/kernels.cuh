@@ -181,9 +181,17 @@ __device__ __forceinline__ void apply_update(float (&p)[VEC], float (&v)[VEC], c
 // state_ptr(0) / state_ptr(1) return the tensor's params / momentum base and are
 // asked again at store time, so that a caller whose bases live in memory need
 // not hold them in registers across the update.
-template <typename G, int VEC, int DEPTH, typename StatePtr, typename GradPtr>
+//
+// after_group(slot, p) is called right after the update of the group that
+// closes on `slot`, with the parameters as they stand then.
+struct NoSnapshot {
+    template <int VEC> __device__ __forceinline__ void operator()(int, int64_t, const float (&)[VEC]) const {}
+};
+
+template <typename G, int VEC, int DEPTH, typename StatePtr, typename GradPtr, typename AfterGroup = NoSnapshot>
 __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first, const FlatSchedule &s,
-                                              const Hyper &h, GradPtr grad_ptr)
+                                              const Hyper &h, GradPtr grad_ptr,
+                                              AfterGroup after_group = AfterGroup())
 {
     constexpr int GB = VEC * G::kBytes;
     float p[VEC], v[VEC], sum[VEC];
@@ -213,6 +221,7 @@ __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first,
                 const int gs = s.group_size[base + j];
                 if (gs == 1) {                       // singleton group: the mean is the gradient
                     apply_update<VEC>(p, v, f, s.neg_lr[base + j], h);
+                    after_group.template operator()<VEC>(base + j, first, p);
                 } else {
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) sum[e] = __fadd_rn(sum[e], f[e]);
@@ -221,6 +230,7 @@ __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first,
 #pragma unroll
                         for (int e = 0; e < VEC; ++e) sum[e] = __fdiv_rn(sum[e], count);
                         apply_update<VEC>(p, v, sum, s.neg_lr[base + j], h);
+                        after_group.template operator()<VEC>(base + j, first, p);
 #pragma unroll
                         for (int e = 0; e < VEC; ++e) sum[e] = -0.0f;
                     }
@@ -261,6 +271,42 @@ star_update_flat_kernel(const __grid_constant__ FlatArgs a)
         const int64_t tail = n_vec * VEC + threadIdx.x;
         if (blockIdx.x == 0 && threadIdx.x < VEC && tail < a.n)
             update_vector<G, 1, DEPTH>(state_ptr, tail, a.sched, a.hyper, grad_ptr);
+    }
+}
+
+// Flat tensor with parameter snapshots: after the update of the group that
+// closes on slot j the parameters are also written to snapshots[j] (if not
+// null) -- the copy the server sends back to that group's workers.
+struct SnapshotArgs {
+    FlatArgs flat;
+    float *snapshots[kMaxWorkers];     // indexed by closing slot
+};
+
+struct StoreSnapshot {
+    const SnapshotArgs *a;
+    template <int VEC> __device__ __forceinline__ void operator()(int slot, int64_t first, const float (&p)[VEC]) const
+    {
+        float *dst = a->snapshots[slot];
+        if (dst != nullptr) store_state<VEC>(dst + first, p);
+    }
+};
+
+template <typename G, int VEC, int DEPTH>
+__global__ void __launch_bounds__(kBlockThreads, kResidentBlocks)
+star_update_flat_snapshot_kernel(const __grid_constant__ SnapshotArgs a)
+{
+    const FlatArgs &f = a.flat;
+    const int64_t n_vec = f.n / VEC;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlockThreads;
+    auto grad_ptr = [&](int slot) -> const void * { return f.grads[f.sched.member[slot]]; };
+    auto state_ptr = [&](int which) -> float * { return which == 0 ? f.params : f.momentum; };
+    const StoreSnapshot snap{&a};
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kBlockThreads + threadIdx.x; i < n_vec; i += stride)
+        update_vector<G, VEC, DEPTH>(state_ptr, i * VEC, f.sched, f.hyper, grad_ptr, snap);
+    if constexpr (VEC > 1) {
+        const int64_t tail = n_vec * VEC + threadIdx.x;
+        if (blockIdx.x == 0 && threadIdx.x < VEC && tail < f.n)
+            update_vector<G, 1, DEPTH>(state_ptr, tail, f.sched, f.hyper, grad_ptr, snap);
     }
 }
 

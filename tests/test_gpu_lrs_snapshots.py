@@ -1,0 +1,106 @@
+"""Per-group learning rates and parameter snapshots (the copy sent back to a
+group's workers) in the fused kernel, against the oracle and closed forms."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import schedule as S
+from oracle import star_oracle as O
+from tests.parity import assert_matches, grad_to_numpy
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2512_09685_b200 import binding
+    return binding
+
+
+def case(n, W, dtype, seed):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    p = torch.randn(n, generator=g, device="cuda") * 0.05
+    v = torch.randn(n, generator=g, device="cuda") * 0.02
+    grads = [(torch.randn(n, generator=g, device="cuda") * 0.01).to(dtype) for _ in range(W)]
+    return p, v, grads
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("n", [1, 7, 4099, 1_000_003])
+def test_lrs_and_snapshots_match_oracle(B, dtype, n):
+    W = 8
+    p, v, grads = case(n, W, dtype, seed=n)
+    off, mem = [0, 3, 4, 6, 8], [5, 0, 2, 7, 1, 3, 4, 6]
+    lrs = [0.1, 0.025, 0.05, 0.2]
+    p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+    g_np = [grad_to_numpy(g) for g in grads]
+    want_snaps = [np.zeros(n, np.float32), None, np.zeros(n, np.float32), np.zeros(n, np.float32)]
+    O.group_update_f32(p_np, v_np, g_np, off, mem, np.array(lrs, np.float32), 0.9, 1e-3, snapshots=want_snaps)
+    snaps = [torch.full((n,), float("nan"), device="cuda"), None,
+             torch.full((n,), float("nan"), device="cuda"), torch.full((n,), float("nan"), device="cuda")]
+    before = B.star_launch_count()
+    B.star_group_update_ex(p, v, grads, off, mem, lrs, 0.9, 1e-3, snapshots=snaps)
+    torch.cuda.synchronize()
+    assert B.star_launch_count() == before + 1
+    assert_matches(p, p_np, "params")
+    assert_matches(v, v_np, "momentum")
+    for k in (0, 2, 3):
+        assert_matches(snaps[k], want_snaps[k], "snapshot %d" % k)
+    assert torch.equal(snaps[3], p)                    # the last group's snapshot is the final state
+
+
+def test_misaligned_snapshot_takes_the_scalar_path(B):
+    n = 5001
+    p, v, grads = case(n, 3, torch.bfloat16, seed=2)
+    p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+    want = [np.zeros(n, np.float32), None]
+    O.group_update_f32(p_np, v_np, [grad_to_numpy(g) for g in grads], [0, 2, 3], [0, 1, 2],
+                       np.array([0.1, 0.2], np.float32), 0.9, 0.0, snapshots=want)
+    snap = torch.empty(n + 1, device="cuda")[1:]
+    B.star_group_update_ex(p, v, grads, [0, 2, 3], [0, 1, 2], [0.1, 0.2], 0.9, 0.0, snapshots=[snap, None])
+    torch.cuda.synchronize()
+    assert_matches(p, p_np, "params")
+    assert_matches(snap, want[0], "snapshot")
+
+
+def test_equal_rates_without_snapshots_equal_the_plain_entry_point(B):
+    n = 77_777
+    p, v, grads = case(n, 6, torch.bfloat16, seed=3)
+    q, u = p.clone(), v.clone()
+    off, mem = [0, 2, 6], [1, 0, 5, 4, 3, 2]
+    B.star_group_update(p, v, grads, off, mem, 0.05, 0.9, 1e-4)
+    B.star_group_update_ex(q, u, grads, off, mem, [0.05, 0.05], 0.9, 1e-4)
+    torch.cuda.synchronize()
+    assert torch.equal(p, q) and torch.equal(v, u)
+
+
+def test_rescaled_rates_make_the_round_schedule_independent(B):
+    """Section IV-C1: r_new = (y / N) r_SSGD.  With mu = wd = 0 every covering
+    schedule then lands on p0 - (r / N) sum_w g_w (up to fp32 rounding)."""
+    n, N, r = 50_000, 8, 0.4
+    p0, _, grads = case(n, N, torch.float32, seed=4)
+    want = p0.double() - (r / N) * sum(g.double() for g in grads)
+    for x in (1, 2, 3, 4, 8):
+        off, mem = B.star_schedule_static_x(None, N, x)
+        lrs = S.scaled_lrs(off, len(off) - 1, N, r)
+        p, v = p0.clone(), torch.zeros(n, device="cuda")
+        B.star_group_update_ex(p, v, grads, off, mem, lrs, 0.0, 0.0)
+        torch.cuda.synchronize()
+        assert float((p.double() - want).abs().max()) <= 16 * 2.0 ** -24 * float(want.abs().max())
+
+
+def test_ex_errors(B):
+    n = 1000
+    p, v, grads = case(n, 2, torch.bfloat16, seed=5)
+    p0 = p.clone()
+    with pytest.raises(B.StarError) as e:              # snapshot overlaps params
+        B.star_group_update_ex(p, v, grads, [0, 2], [0, 1], [0.1], 0.9, 0.0, snapshots=[p])
+    assert e.value.status == B.STAR_ERR_INVALID_ARG
+    s = torch.empty(n, device="cuda")
+    with pytest.raises(B.StarError) as e:              # two groups into one buffer
+        B.star_group_update_ex(p, v, grads, [0, 1, 2], [0, 1], [0.1, 0.1], 0.9, 0.0, snapshots=[s, s])
+    assert e.value.status == B.STAR_ERR_INVALID_ARG
+    with pytest.raises(ValueError):
+        B.star_group_update_ex(p, v, grads, [0, 1, 2], [0, 1], [0.1], 0.9, 0.0)
+    torch.cuda.synchronize()
+    assert torch.equal(p, p0)
