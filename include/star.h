@@ -118,6 +118,50 @@ STAR_API star_status_t star_schedule_dynamic_x(const double *iter_time, const in
                                       int W, int32_t *offsets_out, int32_t *members_out,
                                       int *n_groups_out);
 
+/* ---------------------------------------------------------------------------
+ * Mode decision (host only): from predicted iteration times to the schedule of
+ * the cheapest synchronization mode.  iter_time[w] > 0, finite.
+ * ------------------------------------------------------------------------- */
+
+/* Dynamic x-order clustering (Section IV-B): agglomerative hierarchical
+ * clustering of the W predicted iteration times with average linkage (mean
+ * pairwise |t_a - t_b|).  Merging continues while more than n_clusters clusters
+ * remain (n_clusters <= 0: down to one) and the closest pair is no farther
+ * apart than max_distance (max_distance < 0: no distance limit).  Equally close
+ * pairs: the pair whose clusters hold the smaller worker indices merges first.
+ * cluster_of_worker_out[W] receives labels 0..K-1 numbered by each cluster's
+ * smallest worker index; *n_clusters_out = K.  Feed the labels to
+ * star_schedule_dynamic_x or star_choose_mode. */
+STAR_API star_status_t star_cluster_iteration_times(const double *iter_time, int W, int n_clusters,
+                                                    double max_distance,
+                                                    int32_t *cluster_of_worker_out,
+                                                    int *n_clusters_out);
+
+/* Expected time to a fixed training progress per mode (Section IV-C1).
+ * T_static_out[x-1], x = 1..W, is Eq. 1: (1 + phi / (x M / W)) * t_x, where t_x,
+ * the time one update takes, is read as the x-th smallest iteration time (the
+ * moment x gradient reports are in); x = 1 is ASGD, x = W SSGD.  If
+ * cluster_of_worker is not NULL (labels >= 0 for every worker), *T_dynamic_out
+ * is Eq. 2: 1 / sum_i 1 / ((1 + phi / (n_ci M / W)) * t_ci) over the clusters,
+ * n_ci the cluster's size and t_ci its slowest member.  phi is the
+ * pre-conditioned gradient noise scale of the current update (>= 0), M the
+ * total batch size (> 0); both are the caller's inputs. */
+STAR_API star_status_t star_mode_times(const double *iter_time, const int32_t *cluster_of_worker,
+                                       int W, double phi, double M, double *T_static_out,
+                                       double *T_dynamic_out);
+
+/* The mode with the smallest time and its schedule.  *x_out = x of the chosen
+ * static x-order mode, or 0 for the dynamic mode (only if cluster_of_worker is
+ * given and Eq. 2 is strictly smaller than every Eq. 1 value); equal static
+ * times go to the larger x.  *T_out = that time.  The CSR outputs are as for the
+ * schedule encoders: static modes group the workers in ascending predicted time
+ * (ties by index) in runs of x, members listed in ascending index; the dynamic
+ * mode is star_schedule_dynamic_x on the clusters. */
+STAR_API star_status_t star_choose_mode(const double *iter_time, const int32_t *cluster_of_worker,
+                                        int W, double phi, double M, int *x_out, double *T_out,
+                                        int32_t *offsets_out, int32_t *members_out,
+                                        int *n_groups_out);
+
 /* Sharding helper (host only).  The path is elementwise, so a job spread over
  * several parameter servers / GPUs (the paper runs one to N PSs per job,
  * Section III set-up) needs no exchange inside it: rank r of world owns the

@@ -83,6 +83,13 @@ def _load() -> ctypes.CDLL:
     lib.star_group_update_ex.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
                                          c_vp, c_f, c_f, c_vp, c_vp]
     lib.star_group_update_ex.restype = c_int
+    lib.star_cluster_iteration_times.argtypes = [c_vp, c_int, c_int, ctypes.c_double, c_vp, c_vp]
+    lib.star_cluster_iteration_times.restype = c_int
+    lib.star_mode_times.argtypes = [c_vp, c_vp, c_int, ctypes.c_double, ctypes.c_double, c_vp, c_vp]
+    lib.star_mode_times.restype = c_int
+    lib.star_choose_mode.argtypes = [c_vp, c_vp, c_int, ctypes.c_double, ctypes.c_double, c_vp, c_vp,
+                                     c_vp, c_vp, c_vp]
+    lib.star_choose_mode.restype = c_int
     lib.star_shard_range.argtypes = [c_i64, c_int, c_int, c_i64, c_vp, c_vp]
     lib.star_shard_range.restype = c_int
     lib.star_host_workspace_bytes.argtypes = [c_int, c_int, c_i64, c_vp]
@@ -173,6 +180,43 @@ def star_schedule_dynamic_x(iter_time: Sequence[float], cluster_of_worker: Seque
     _check(_lib.star_schedule_dynamic_x(times, _i32(cluster_of_worker), W, offsets, members,
                                         ctypes.byref(K)), "star_schedule_dynamic_x")
     return _unpack(offsets, members, K)
+
+
+def _f64(values: Sequence[float]):
+    return (ctypes.c_double * max(len(values), 1))(*values)
+
+
+def star_cluster_iteration_times(iter_time: Sequence[float], n_clusters: int = 0,
+                                 max_distance: float = -1.0) -> List[int]:
+    """Cluster label per worker (average-linkage agglomerative clustering)."""
+    W = len(iter_time)
+    labels, K = _i32([0] * W), ctypes.c_int(0)
+    _check(_lib.star_cluster_iteration_times(_f64(iter_time), W, n_clusters, max_distance, labels,
+                                             ctypes.byref(K)), "star_cluster_iteration_times")
+    return list(labels[:W])
+
+
+def star_mode_times(iter_time: Sequence[float], cluster_of_worker: Optional[Sequence[int]], phi: float,
+                    M: float) -> Tuple[List[float], Optional[float]]:
+    """(T_x for x = 1..W by Eq. 1, T_d by Eq. 2 or None without clusters)."""
+    W = len(iter_time)
+    T_static, T_dynamic = _f64([0.0] * W), ctypes.c_double(0.0)
+    clusters = None if cluster_of_worker is None else _i32(cluster_of_worker)
+    _check(_lib.star_mode_times(_f64(iter_time), clusters, W, phi, M, T_static, ctypes.byref(T_dynamic)),
+           "star_mode_times")
+    return list(T_static[:W]), (None if clusters is None else T_dynamic.value)
+
+
+def star_choose_mode(iter_time: Sequence[float], cluster_of_worker: Optional[Sequence[int]], phi: float,
+                     M: float) -> Tuple[int, float, Schedule]:
+    """(x, T, schedule): x = 0 means the dynamic mode."""
+    W = len(iter_time)
+    x, T, K = ctypes.c_int(0), ctypes.c_double(0.0), ctypes.c_int(0)
+    offsets, members = _i32([0] * (W + 1)), _i32([0] * W)
+    clusters = None if cluster_of_worker is None else _i32(cluster_of_worker)
+    _check(_lib.star_choose_mode(_f64(iter_time), clusters, W, phi, M, ctypes.byref(x), ctypes.byref(T),
+                                 offsets, members, ctypes.byref(K)), "star_choose_mode")
+    return x.value, T.value, _unpack(offsets, members, K)
 
 
 def star_shard_range(n: int, world: int, rank: int, align: int = 16) -> Tuple[int, int]:

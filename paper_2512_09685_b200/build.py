@@ -16,7 +16,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libstar.so")
-SOURCES = ["api.cu", "schedule.cc"]
+SOURCES = ["api.cu", "schedule.cc", "mode_decision.cc"]
 HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(ROOT, "include", "star.h")]
 
 NVCC_FLAGS = [

@@ -1,0 +1,76 @@
+"""The library's host-side mode decision against the Python oracle."""
+import random
+
+import pytest
+
+from oracle import mode_decision as D
+from oracle import schedule as S
+from paper_2512_09685_b200 import binding as B
+
+
+def test_clustering_matches_oracle():
+    rng = random.Random(0)
+    for trial in range(200):
+        W = rng.randint(1, 14)
+        t = [rng.choice([0.2, 0.25, 0.5, 1.0]) + rng.random() * rng.choice([0.0, 0.01, 0.2]) for _ in range(W)]
+        if trial % 7 == 0:
+            t = [rng.choice([0.2, 0.4, 0.8]) for _ in range(W)]           # exact ties
+        for k in (0, 1, 2, 3, W):
+            assert B.star_cluster_iteration_times(t, k, -1.0) == D.agglomerative_clusters(t, n_clusters=k or None)
+        for thr in (0.0, 0.05, 0.3):
+            assert B.star_cluster_iteration_times(t, 0, thr) == D.agglomerative_clusters(t, max_distance=thr)
+            assert B.star_cluster_iteration_times(t, 2, thr) == \
+                D.agglomerative_clusters(t, n_clusters=2, max_distance=thr)
+
+
+def test_mode_times_and_choice_match_oracle():
+    rng = random.Random(1)
+    chosen = set()
+    for _ in range(300):
+        W = rng.randint(1, 16)
+        t = [rng.uniform(0.1, 0.5) * rng.choice([1, 1, 1, 4]) for _ in range(W)]
+        labels = D.agglomerative_clusters(t, max_distance=0.1)
+        phi, M = rng.choice([0.0, 10.0, 500.0, 1e5]), rng.choice([128.0, 1024.0])
+        T_static, T_dynamic = B.star_mode_times(t, labels, phi, M)
+        for x in range(1, W + 1):
+            assert T_static[x - 1] == pytest.approx(D.time_static_x(t, x, phi, M), rel=1e-14)
+        assert T_dynamic == pytest.approx(D.time_dynamic(t, labels, phi, M), rel=1e-14)
+        x, T, (off, mem) = B.star_choose_mode(t, labels, phi, M)
+        want_x, want_T = D.choose_mode(t, labels, phi, M)
+        assert x == want_x and T == pytest.approx(want_T, rel=1e-14)
+        chosen.add(min(x, 2) if x < W else "ssgd")
+        if x == 0:
+            assert (off, mem) == tuple(S.dynamic_x(t, labels))
+        else:
+            order = sorted(range(W), key=lambda w: (t[w], w))
+            assert (off, mem) == tuple(S.static_x(order, W, x, sort_members=True))
+        assert B.star_schedule_validate(off, mem, len(off) - 1, W) == B.STAR_OK
+    assert len(chosen) >= 3                                     # dynamic, low-order and SSGD all occur
+
+
+def test_worked_example_through_the_library():
+    t = [1.0, 1.0, 2.0, 4.0]
+    labels = B.star_cluster_iteration_times(t, 3)
+    assert labels == [0, 0, 1, 2]
+    T_static, T_dynamic = B.star_mode_times(t, labels, 64.0, 128.0)
+    assert T_static == pytest.approx([3.0, 2.0, 10 / 3, 6.0]) and T_dynamic == pytest.approx(4 / 3)
+    x, T, (off, mem) = B.star_choose_mode(t, labels, 64.0, 128.0)
+    assert x == 0 and (off, mem) == ([0, 2, 3, 4], [0, 1, 2, 3])
+    x, T, sched = B.star_choose_mode(t, None, 64.0, 128.0)      # without clusters: best static mode
+    assert x == 2 and T == pytest.approx(2.0) and sched == ([0, 2, 4], [0, 1, 2, 3])
+
+
+def test_mode_decision_rejects_bad_input():
+    for t in ([0.0, 1.0], [-1.0, 1.0], [float("nan"), 1.0], [float("inf"), 1.0]):
+        with pytest.raises(B.StarError):
+            B.star_cluster_iteration_times(t, 1)
+        with pytest.raises(B.StarError):
+            B.star_mode_times(t, None, 1.0, 64.0)
+    with pytest.raises(B.StarError):
+        B.star_mode_times([1.0, 2.0], None, -1.0, 64.0)
+    with pytest.raises(B.StarError):
+        B.star_mode_times([1.0, 2.0], None, 1.0, 0.0)
+    with pytest.raises(B.StarError):
+        B.star_mode_times([1.0, 2.0], [0, -1], 1.0, 64.0)
+    with pytest.raises(B.StarError):
+        B.star_choose_mode([], None, 1.0, 64.0)

@@ -1,0 +1,88 @@
+"""Pins for the mode-decision oracle: a hand-worked example of Eq. 1 / Eq. 2,
+identities between the two equations, and SciPy's hierarchical clustering."""
+import os
+
+import numpy as np
+import pytest
+from scipy.cluster.hierarchy import fcluster, linkage
+
+from oracle import mode_decision as D
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "mode_decision_example.txt")
+
+
+def read_golden():
+    out = {}
+    for line in open(GOLDEN):
+        if line.startswith("#") or not line.strip():
+            continue
+        key, *vals = line.split()
+        out[key] = [float(v) for v in vals]
+    return out
+
+
+def test_hand_worked_example():
+    g = read_golden()
+    t, M, phi = g["t"], g["M"][0], g["phi"][0]
+    labels = [int(c) for c in g["clusters"]]
+    for x, want in enumerate(g["T_static"], start=1):
+        assert D.time_static_x(t, x, phi, M) == pytest.approx(want, rel=1e-14)
+    assert D.time_dynamic(t, labels, phi, M) == pytest.approx(g["T_dynamic"][0], rel=1e-14)
+    x, T = D.choose_mode(t, labels, phi, M)
+    assert x == int(g["best_x"][0]) and T == pytest.approx(4 / 3, rel=1e-14)
+    assert D.agglomerative_clusters(t, n_clusters=3) == labels
+
+
+def test_eq2_with_one_cluster_is_eq1_at_x_equal_n():
+    t = [0.3, 0.5, 0.25, 0.9, 0.4]
+    assert D.time_dynamic(t, [0] * 5, 10.0, 640.0) == pytest.approx(D.time_static_x(t, 5, 10.0, 640.0))
+    # SSGD: (1 + phi / M) * slowest worker
+    assert D.time_static_x(t, 5, 10.0, 640.0) == pytest.approx((1 + 10 / 640) * 0.9)
+
+
+def test_equal_workers_closed_form():
+    """No stragglers, all N workers take t: T_x = (1 + phi N / (x M)) t falls with
+    x, so SSGD is chosen (Section IV-B: a higher order has the lower TTA)."""
+    N, t, M = 8, 0.2, 1024.0
+    for phi in (1.0, 1e5):
+        for x in range(1, N + 1):
+            assert D.time_static_x([t] * N, x, phi, M) == pytest.approx((1 + phi * N / (x * M)) * t)
+        assert D.choose_mode([t] * N, [0] * N, phi, M)[0] == N
+
+
+def test_order_statistics_define_t_x():
+    t = [0.7, 0.2, 0.9, 0.4]
+    for x, want in zip((1, 2, 3, 4), (0.2, 0.4, 0.7, 0.9)):
+        assert D.time_static_x(t, x, 0.0, 64.0) == pytest.approx(want)       # phi = 0: T_x = t_x
+
+
+def test_a_straggler_pushes_the_choice_away_from_ssgd():
+    t = [0.2] * 7 + [2.0]                      # one worker ten times slower
+    labels = D.agglomerative_clusters(t, max_distance=0.1)
+    assert labels == [0] * 7 + [1]
+    x, T = D.choose_mode(t, labels, 2000.0, 1024.0)
+    assert x == 0                              # dynamic: the seven fast workers synchronize among themselves
+    assert T < D.time_static_x(t, 7, 2000.0, 1024.0) < D.time_static_x(t, 8, 2000.0, 1024.0)
+
+
+def canonical(labels):
+    seen, out = {}, []
+    for l in labels:
+        seen.setdefault(l, len(seen))
+        out.append(seen[l])
+    return out
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_clustering_matches_scipy_average_linkage(seed):
+    rng = np.random.default_rng(seed)
+    N = int(rng.integers(2, 17))
+    t = rng.uniform(0.1, 1.0, N) + rng.choice([0.0, 1.0, 3.0], N)       # clumpy
+    Z = linkage(t.reshape(-1, 1), method="average", metric="euclidean")
+    for k in range(1, N + 1):
+        want = canonical(fcluster(Z, k, criterion="maxclust"))
+        got = D.agglomerative_clusters(list(t), n_clusters=k)
+        assert got == want, (k, list(t))
+    for thr in (0.05, 0.3, 1.5):
+        want = canonical(fcluster(Z, thr, criterion="distance"))
+        assert D.agglomerative_clusters(list(t), max_distance=thr) == want
