@@ -43,8 +43,12 @@ struct Hyper {
 };
 
 // ---------------------------------------------------------------------------
-// Memory operations.  Gradients are read exactly once: non-coherent path, no
-// L1 allocation.  p and v are read once and written once.
+// Memory operations.  Gradients are read exactly once through the read-only
+// (non-coherent) path with the default L1 policy: measured on B200 this is
+// 2.5-6 % faster than the same loads with L1::no_allocate, evict-first or
+// last-use hints (6445 vs 6280 GB/s on the ResNet-50-sized round, 6890 vs 6500
+// on the 32-worker ASGD round).  p and v are read once and written once; their
+// cache hints made no measurable difference.
 // ---------------------------------------------------------------------------
 template <int BYTES> struct Raw;              // BYTES of payload in 32-bit registers
 template <> struct Raw<2>  { uint32_t w[1]; };
@@ -58,20 +62,20 @@ template <> __device__ __forceinline__ Raw<2> load_stream<2>(const void *p)
 {
     Raw<2> r;
     unsigned short h;
-    asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(h) : "l"(p));
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(h) : "l"(p));
     r.w[0] = h;
     return r;
 }
 template <> __device__ __forceinline__ Raw<4> load_stream<4>(const void *p)
 {
     Raw<4> r;
-    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(r.w[0]) : "l"(p));
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(r.w[0]) : "l"(p));
     return r;
 }
 template <> __device__ __forceinline__ Raw<16> load_stream<16>(const void *p)
 {
     Raw<16> r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p));
     return r;
 }
