@@ -406,8 +406,9 @@ def main():
     ap.add_argument("--workload", default=HEADLINE)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--n", type=int, default=0,
-                    help="run a flat workload at this many elements instead of its full size "
-                         "(small cases for profiler captures; not a benchmark configuration)")
+                    help="run the workload at a reduced size (flat: this many elements; tensor list: 2 "
+                         "layers and n/1024 vocabulary rows): small cases for profiler captures, "
+                         "not a benchmark configuration")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-extra", action="store_true",
                     help="device-timed headline only: skip the end-to-end leg, the other workloads "
@@ -439,7 +440,9 @@ def main():
 
     w = WL.BY_NAME[args.workload]
     if args.n > 0:
-        w = WL.scaled(w, args.n)
+        # reduced sizes for profiler captures: a flat workload at n elements, the
+        # tensor list with 2 layers and a vocabulary of n / 1024 rows
+        w = WL.reduced_list(w, 2, max(args.n // 1024, 1)) if w.multi_tensor else WL.scaled(w, args.n)
     peak, peak_kind = measured_peak()
     dw = DeviceWorkload(w, grad_sets=2 if w.n * w.W * w.grad_bytes < (4 << 30) else 1)
     sampler = ClockSampler(local_rank)

@@ -165,10 +165,11 @@ class Workload:
         return self.n * (scheduled_workers * self.grad_bytes + 16)
 
 
-def gpt2_medium_shapes() -> Tuple[Tuple[str, Tuple[int, ...]], ...]:
+def gpt2_medium_shapes(layers: int = 24, vocab: int = 50257) -> Tuple[Tuple[str, Tuple[int, ...]], ...]:
     """The 292 parameter tensors of a GPT-2-medium-shaped model: d=1024, 24
-    layers, vocabulary 50257, 1024 positions, tied output head."""
-    d, layers, vocab, positions = 1024, 24, 50257, 1024
+    layers, vocabulary 50257, 1024 positions, tied output head.  Fewer layers
+    or a smaller vocabulary give a shorter list of the same kinds of tensors."""
+    d, positions = 1024, 1024
     shapes: List[Tuple[str, Tuple[int, ...]]] = [("wte", (vocab, d)), ("wpe", (positions, d))]
     for l in range(layers):
         pre = "h%d." % l
@@ -208,6 +209,12 @@ def scaled(workload: Workload, n: int) -> Workload:
     """The same workload on a flat tensor of ``n`` elements (for small parity
     cases and bounded CPU samples)."""
     return dataclasses.replace(workload, shapes=_flat("flat", n), multi_tensor=False)
+
+
+def reduced_list(workload: Workload, layers: int, vocab: int) -> Workload:
+    """A tensor-list workload with the same tensor kinds but fewer layers and a
+    smaller vocabulary (small cases for profiler captures)."""
+    return dataclasses.replace(workload, shapes=gpt2_medium_shapes(layers, vocab))
 
 
 def _generator(device, seed: int) -> torch.Generator:
