@@ -302,53 +302,69 @@ def time_e2e(w, steps: int, warmup: int, dist):
 # ---------------------------------------------------------------------------
 # CPU oracle timing
 # ---------------------------------------------------------------------------
-def time_oracle(w, n_sample: int, min_seconds: float, threads: int):
-    """The oracle, as it stands, on the first `n_sample` elements of workload
-    `w` (inputs generated on the CPU), `threads` Python threads over disjoint
-    index ranges (the C call releases the GIL).  Returns (GB/s, elements/s,
-    rounds run, seconds)."""
-    import numpy as np
-    import torch
-    from oracle import schedule as S
-    from oracle import star_oracle as O
-    from paper_2512_09685_b200 import workloads as WL
+class OracleRunner:
+    """The CPU oracle, as it stands, on the first `n_sample` elements of a
+    workload (inputs generated once on the CPU), `threads` Python threads over
+    disjoint index ranges (the C call releases the GIL)."""
 
-    ws = WL.scaled(w, n_sample)
-    p = WL.make_params(ws, "cpu")[0].numpy()
-    v = WL.make_momentum(ws, "cpu")[0].numpy()
-    grads = []
-    for g in WL.make_grads(ws, 0, "cpu"):
-        g = g[0]
-        grads.append(g.view(torch.int16).numpy().view(np.uint16) if g.dtype == torch.bfloat16 else g.numpy())
-    bounds = [n_sample * i // threads for i in range(threads + 1)]
+    def __init__(self, w, n_sample: int, threads: int):
+        import numpy as np
+        import torch
+        from oracle import schedule as S
+        from oracle import star_oracle as O
+        from paper_2512_09685_b200 import workloads as WL
+        self.np, self.S, self.O, self.w = np, S, O, w
+        self.n, self.threads = n_sample, threads
+        ws = WL.scaled(w, n_sample)
+        self.p = WL.make_params(ws, "cpu")[0].numpy()
+        self.v = WL.make_momentum(ws, "cpu")[0].numpy()
+        self.grads = []
+        for g in WL.make_grads(ws, 0, "cpu"):
+            g = g[0]
+            self.grads.append(g.view(torch.int16).numpy().view(np.uint16) if g.dtype == torch.bfloat16
+                              else g.numpy())
+        self.rounds_done = 0
+        O.build()
 
-    def encode(step):
-        d = w.decision(step)
+    def encode(self, step):
+        d = self.w.decision(step)
         if d.kind == "labels":
-            return S.from_labels(d.labels)
-        return S.static_x(d.arrival_order, d.W, d.x, d.sort_members)
+            return self.S.from_labels(d.labels)
+        return self.S.static_x(d.arrival_order, d.W, d.x, d.sort_members)
 
-    def one_round(step):
-        off, mem = encode(step)
-        lr = np.float32(w.lr)
+    def round(self, n=None) -> int:
+        """One round on the first n (default: all sampled) elements; returns the
+        number of scheduled workers."""
+        n = self.n if n is None else n
+        off, mem = self.encode(self.rounds_done)
+        self.rounds_done += 1
+        w, lr = self.w, self.np.float32(self.w.lr)
+        bounds = [n * i // self.threads for i in range(self.threads + 1)]
+
         def work(i):
             a, b = bounds[i], bounds[i + 1]
-            O.group_update_f32(p[a:b], v[a:b], [g[a:b] for g in grads], off, mem, lr, w.mu, w.wd)
-        if threads == 1:
+            self.O.group_update_f32(self.p[a:b], self.v[a:b], [g[a:b] for g in self.grads], off, mem,
+                                    lr, w.mu, w.wd)
+        if self.threads == 1:
             work(0)
         else:
-            ts = [threading.Thread(target=work, args=(i,)) for i in range(threads)]
+            ts = [threading.Thread(target=work, args=(i,)) for i in range(self.threads)]
             for t in ts:
                 t.start()
             for t in ts:
                 t.join()
         return off[-1]
 
-    one_round(0)                                   # warm-up (also builds the oracle)
+
+def time_oracle(w, n_sample: int, min_seconds: float, threads: int):
+    """Rounds of the oracle for at least `min_seconds`.  Returns (GB/s,
+    elements/s, rounds run, seconds)."""
+    runner = OracleRunner(w, n_sample, threads)
+    runner.round()                                 # warm-up
     rounds, scheduled = 0, 0
     t0 = time.perf_counter()
     while True:
-        scheduled += one_round(rounds + 1)
+        scheduled += runner.round()
         rounds += 1
         dt = time.perf_counter() - t0
         if dt >= min_seconds:
@@ -365,32 +381,43 @@ def host_cores() -> int:
 
 
 # ---------------------------------------------------------------------------
+REFERENCE_BUDGET_SECONDS = 100.0
+
+
 def run_reference(args, rank: int):
-    """--impl reference: the CPU oracle on the host cores."""
+    """--impl reference: the CPU oracle on the host cores.  A step is one round on
+    a bounded sample of the workload: the first n_sample elements, n_sample
+    chosen from a calibration round so that warm-up + steps fit the budget."""
     if rank != 0:
         return
     from paper_2512_09685_b200 import workloads as WL
     w = WL.BY_NAME[args.workload]
     cores = host_cores()
-    n_sample = min(w.n, 4_000_000)
-    per_step = []
-    for _ in range(max(args.warmup, 0)):
-        time_oracle(w, n_sample, 0.0, cores)
+    runner = OracleRunner(w, w.n if w.n <= 32_000_000 else 32_000_000, cores)
+    probe = min(runner.n, 2_000_000)
+    runner.round(probe)
     t0 = time.perf_counter()
-    gbs_acc = []
+    runner.round(probe)
+    rate = probe / (time.perf_counter() - t0)                        # elements / s
+    total_rounds = max(args.steps, 1) + max(args.warmup, 0)
+    n_sample = int(min(runner.n, max(65_536, rate * REFERENCE_BUDGET_SECONDS / total_rounds)))
+    for _ in range(max(args.warmup, 0)):
+        runner.round(n_sample)
+    scheduled = 0
+    t0 = time.perf_counter()
     for _ in range(args.steps):
-        gbs, eps, rounds, dt = time_oracle(w, n_sample, 0.0, cores)
-        gbs_acc.append(gbs)
-        per_step.append(dt / rounds * 1e3)
-    value = statistics.mean(gbs_acc)
+        scheduled += runner.round(n_sample)
+    seconds = time.perf_counter() - t0
+    value = n_sample * (scheduled * w.grad_bytes + 16 * args.steps) / seconds / 1e9
     sample = "first %d of %d elements of %s per step, %d threads over disjoint ranges" % (
         n_sample, w.n, w.name, cores)
     out = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": statistics.mean(per_step),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": seconds / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "config": {"workload": w.name, "model": w.model, "n": w.n, "W": w.W,
                                         "grad_dtype": w.grad_dtype, "sample_elements": n_sample},
+        "param_elements_per_s": n_sample * args.steps / seconds,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
