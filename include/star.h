@@ -72,6 +72,15 @@ typedef enum {
 
 typedef enum { STAR_DTYPE_F32 = 0, STAR_DTYPE_BF16 = 1 } star_dtype_t;
 
+/* Order of the additions inside a group (only rounding depends on it).
+ * STAR_SUM_LINEAR: left to right in the listed member order.
+ * STAR_SUM_TREE:   pairwise, as gradients are combined along a binary
+ *                  aggregation tree (Section IV-D2b: workers add their children's
+ *                  gradients to their own on the way up): tree(m_0..m_{c-1}) is the
+ *                  member itself for c = 1, else tree(first h) + tree(remaining
+ *                  c - h) with h the largest power of two below c. */
+typedef enum { STAR_SUM_LINEAR = 0, STAR_SUM_TREE = 1 } star_sum_order_t;
+
 #define STAR_MAX_WORKERS 64
 
 /* Static, NUL-terminated name of a status code. */
@@ -187,8 +196,10 @@ STAR_API star_status_t star_group_update(float *params, float *momentum, const v
                                 const int32_t *group_offsets, const int32_t *group_members,
                                 int n_groups, float lr, float mu, float wd, void *cuda_stream);
 
-/* The same round with one learning rate per group and optional parameter
- * snapshots.
+/* The same round with one learning rate per group, optional parameter
+ * snapshots and a choice of the in-group summation order (sum_order; the tree
+ * order runs at two resident blocks per SM instead of four and is somewhat
+ * slower).
  *   lrs        : host, n_groups learning rates.  Section IV-C1 ("Scaling learning
  *                rate after switching") sets the rate of an update built from y
  *                gradient reports to (y / N) x the SSGD rate; the caller computes
@@ -206,7 +217,8 @@ STAR_API star_status_t star_group_update_ex(float *params, float *momentum, cons
                                             const int32_t *group_offsets,
                                             const int32_t *group_members, int n_groups,
                                             const float *lrs, float mu, float wd,
-                                            float *const *snapshots, void *cuda_stream);
+                                            float *const *snapshots, star_sum_order_t sum_order,
+                                            void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
  * Fused grouped update of a LIST of tensors (per-layer parameters) in one

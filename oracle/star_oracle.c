@@ -33,6 +33,14 @@
  *         v[i] = mu * v[i] + d
  *         p[i] = p[i] - lr * v[i]
  *
+ * In-group summation order (sum_order argument):
+ *   0  linear: left to right in the listed member order (the default reading).
+ *   1  tree:   pairwise, as gradients are combined along a binary aggregation
+ *              tree (Section IV-D2b, workers add their children's gradients to
+ *              their own on the way up): tree(m_0..m_{c-1}) = the member itself
+ *              for c = 1, otherwise tree(first h) + tree(remaining c - h) with
+ *              h the largest power of two below c.
+ *
  * Two variants:
  *   oracle_group_update_f32  canonical binary32 sequence; each line above is
  *                            ONE correctly rounded IEEE operation: fp32 add,
@@ -69,6 +77,27 @@ static float grad_at(const void *buf, int dtype, int64_t i)
     if (dtype == ORACLE_DTYPE_BF16)
         return widen_bf16(((const uint16_t *)buf)[i]);
     return ((const float *)buf)[i];
+}
+
+/* Pairwise (tree) sum of members[0..count) at element i, binary32. */
+static float tree_sum_f32(const void *const *grads, int dtype, const int32_t *members, int count, int64_t i)
+{
+    if (count == 1)
+        return grad_at(grads[members[0]], dtype, i);
+    int h = 1;
+    while (2 * h < count)
+        h *= 2;
+    return tree_sum_f32(grads, dtype, members, h, i) + tree_sum_f32(grads, dtype, members + h, count - h, i);
+}
+
+static double tree_sum_f64(const void *const *grads, int dtype, const int32_t *members, int count, int64_t i)
+{
+    if (count == 1)
+        return (double)grad_at(grads[members[0]], dtype, i);
+    int h = 1;
+    while (2 * h < count)
+        h *= 2;
+    return tree_sum_f64(grads, dtype, members, h, i) + tree_sum_f64(grads, dtype, members + h, count - h, i);
 }
 
 /* 1 if the schedule is one the definition covers, else 0.  The public
@@ -108,9 +137,9 @@ int oracle_group_update_f32(float *params, float *momentum,
                             int64_t n, const int32_t *group_offsets,
                             const int32_t *group_members, int n_groups,
                             const float *lrs, float mu, float wd,
-                            float *const *snapshots)
+                            float *const *snapshots, int sum_order)
 {
-    if (!schedule_ok(group_offsets, group_members, n_groups, W))
+    if (!schedule_ok(group_offsets, group_members, n_groups, W) || sum_order < 0 || sum_order > 1)
         return 1;
     for (int64_t i = 0; i < n; ++i) {
         float p = params[i];
@@ -118,9 +147,14 @@ int oracle_group_update_f32(float *params, float *momentum,
         for (int k = 0; k < n_groups; ++k) {
             const int first = group_offsets[k];
             const int last = group_offsets[k + 1];
-            float s = grad_at(grads[group_members[first]], grad_dtype, i);
-            for (int j = first + 1; j < last; ++j)
-                s = s + grad_at(grads[group_members[j]], grad_dtype, i);
+            float s;
+            if (sum_order == 1) {
+                s = tree_sum_f32(grads, grad_dtype, group_members + first, last - first, i);
+            } else {
+                s = grad_at(grads[group_members[first]], grad_dtype, i);
+                for (int j = first + 1; j < last; ++j)
+                    s = s + grad_at(grads[group_members[j]], grad_dtype, i);
+            }
             const float gbar = s / (float)(last - first);
             const float d = fmaf(wd, p, gbar);
             v = fmaf(mu, v, d);
@@ -140,9 +174,9 @@ int oracle_group_update_f64(double *params, double *momentum,
                             int64_t n, const int32_t *group_offsets,
                             const int32_t *group_members, int n_groups,
                             const double *lrs, double mu, double wd,
-                            double *const *snapshots)
+                            double *const *snapshots, int sum_order)
 {
-    if (!schedule_ok(group_offsets, group_members, n_groups, W))
+    if (!schedule_ok(group_offsets, group_members, n_groups, W) || sum_order < 0 || sum_order > 1)
         return 1;
     for (int64_t i = 0; i < n; ++i) {
         double p = params[i];
@@ -150,9 +184,14 @@ int oracle_group_update_f64(double *params, double *momentum,
         for (int k = 0; k < n_groups; ++k) {
             const int first = group_offsets[k];
             const int last = group_offsets[k + 1];
-            double s = (double)grad_at(grads[group_members[first]], grad_dtype, i);
-            for (int j = first + 1; j < last; ++j)
-                s = s + (double)grad_at(grads[group_members[j]], grad_dtype, i);
+            double s;
+            if (sum_order == 1) {
+                s = tree_sum_f64(grads, grad_dtype, group_members + first, last - first, i);
+            } else {
+                s = (double)grad_at(grads[group_members[first]], grad_dtype, i);
+                for (int j = first + 1; j < last; ++j)
+                    s = s + (double)grad_at(grads[group_members[j]], grad_dtype, i);
+            }
             const double gbar = s / (double)(last - first);
             const double d = gbar + wd * p;
             v = mu * v + d;

@@ -51,10 +51,10 @@ def _load():
                   ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
                   ctypes.c_int, ctypes.c_void_p]
         lib.oracle_group_update_f32.argtypes = common + [
-            ctypes.c_float, ctypes.c_float, ctypes.c_void_p]
+            ctypes.c_float, ctypes.c_float, ctypes.c_void_p, ctypes.c_int]
         lib.oracle_group_update_f32.restype = ctypes.c_int
         lib.oracle_group_update_f64.argtypes = common + [
-            ctypes.c_double, ctypes.c_double, ctypes.c_void_p]
+            ctypes.c_double, ctypes.c_double, ctypes.c_void_p, ctypes.c_int]
         lib.oracle_group_update_f64.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -69,8 +69,11 @@ def _grad_dtype(grads: Sequence[Optional[np.ndarray]]) -> int:
     raise TypeError("gradients must all be float32, or all uint16 (bf16 bits): %r" % kinds)
 
 
+SUM_ORDERS = {"linear": 0, "tree": 1}
+
+
 def _call(fn, real, params, momentum, grads, group_offsets, group_members, lrs, mu, wd,
-          snapshots):
+          snapshots, sum_order="linear"):
     n = params.shape[0]
     if params.dtype != real or momentum.dtype != real:
         raise TypeError("params/momentum must be %s" % real)
@@ -112,26 +115,27 @@ def _call(fn, real, params, momentum, grads, group_offsets, group_members, lrs, 
             snap_ptrs[k] = s.ctypes.data
     rc = fn(params.ctypes.data, momentum.ctypes.data, ptrs, W, dt, n,
             off.ctypes.data, mem.ctypes.data, K, lr_arr.ctypes.data,
-            mu, wd, snap_ptrs)
+            mu, wd, snap_ptrs, SUM_ORDERS[sum_order])
     if rc != 0:
         raise ValueError("schedule outside the definition (empty group, duplicate or "
                          "out-of-range member)")
 
 
 def group_update_f32(params, momentum, grads, group_offsets, group_members, lrs, mu, wd,
-                     snapshots=None):
+                     snapshots=None, sum_order="linear"):
     """Canonical binary32 grouped update, in place on ``params`` / ``momentum``.
 
     ``lrs`` is a scalar or one learning rate per group.  ``mu`` and ``wd`` are
     rounded to binary32 on the way in, as the C signature takes floats.
+    ``sum_order`` is "linear" (left to right) or "tree" (pairwise).
     """
     _call(_load().oracle_group_update_f32, np.float32, params, momentum, grads,
           group_offsets, group_members, lrs, float(np.float32(mu)), float(np.float32(wd)),
-          snapshots)
+          snapshots, sum_order)
 
 
 def group_update_f64(params, momentum, grads, group_offsets, group_members, lrs, mu, wd,
-                     snapshots=None):
+                     snapshots=None, sum_order="linear"):
     """Binary64 shadow of the same loop, in place on float64 arrays."""
     _call(_load().oracle_group_update_f64, np.float64, params, momentum, grads,
-          group_offsets, group_members, lrs, float(mu), float(wd), snapshots)
+          group_offsets, group_members, lrs, float(mu), float(wd), snapshots, sum_order)

@@ -31,6 +31,8 @@ STAR_ERR_CUDA = 6
 STAR_DTYPE_F32 = 0
 STAR_DTYPE_BF16 = 1
 STAR_MAX_WORKERS = 64
+STAR_SUM_LINEAR = 0
+STAR_SUM_TREE = 1
 
 
 class StarError(RuntimeError):
@@ -81,7 +83,7 @@ def _load() -> ctypes.CDLL:
                                        ctypes.c_size_t, c_vp, c_vp]
     lib.star_group_update_multi.argtypes = [c_vp, c_vp, c_vp, c_int, c_f, c_f, c_f, c_vp]
     lib.star_group_update_ex.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
-                                         c_vp, c_f, c_f, c_vp, c_vp]
+                                         c_vp, c_f, c_f, c_vp, c_int, c_vp]
     lib.star_group_update_ex.restype = c_int
     lib.star_cluster_iteration_times.argtypes = [c_vp, c_int, c_int, ctypes.c_double, c_vp, c_vp]
     lib.star_cluster_iteration_times.restype = c_int
@@ -293,9 +295,10 @@ def star_group_update_ex(params: torch.Tensor, momentum: torch.Tensor,
                          grads: Sequence[Optional[torch.Tensor]], group_offsets: Sequence[int],
                          group_members: Sequence[int], lrs: Sequence[float], mu: float, wd: float,
                          snapshots: Optional[Sequence[Optional[torch.Tensor]]] = None,
-                         stream=None) -> None:
+                         sum_order: int = STAR_SUM_LINEAR, stream=None) -> None:
     """The round with one learning rate per group; ``snapshots[k]`` (fp32 CUDA
-    tensor or None) receives the parameters right after group k's update."""
+    tensor or None) receives the parameters right after group k's update;
+    ``sum_order`` is STAR_SUM_LINEAR or STAR_SUM_TREE."""
     n = params.numel()
     p, v = _state(params, "params"), _state(momentum, "momentum")
     if momentum.numel() != n:
@@ -330,7 +333,7 @@ def star_group_update_ex(params: torch.Tensor, momentum: torch.Tensor,
             snap_arr[k] = _state(s, "snapshot")
     _check(_lib.star_group_update_ex(p, v, ptrs, W, STAR_DTYPE_F32 if dt is None else dt, n,
                                      _i32(group_offsets), _i32(group_members), K, lr_arr, mu, wd,
-                                     snap_arr, _stream(stream)), "star_group_update_ex")
+                                     snap_arr, sum_order, _stream(stream)), "star_group_update_ex")
 
 
 def star_multi_workspace_bytes(sizes: Sequence[int], W: int) -> int:

@@ -76,10 +76,11 @@ int choose_grid(int64_t work, int resident)
 }
 
 // ---------------------------------------------------------------------------
-// Schedule: validate, then flatten into the kernel's slot list.
+// Schedule: validate, then flatten into the kernel's slot list.  lrs (one rate
+// per group) overrides the single rate lr when given.
 // ---------------------------------------------------------------------------
 star_status_t flatten_schedule(const int32_t *group_offsets, const int32_t *group_members, int n_groups,
-                               int W, float lr, FlatSchedule *out, const float *lrs = nullptr)
+                               int W, float lr, FlatSchedule *out, const float *lrs)
 {
     const star_status_t st = star_schedule_validate(group_offsets, group_members, n_groups, W);
     if (st != STAR_OK) return st;
@@ -87,7 +88,10 @@ star_status_t flatten_schedule(const int32_t *group_offsets, const int32_t *grou
     out->n_slots = n_groups > 0 ? group_offsets[n_groups] : 0;
     for (int k = 0; k < n_groups; ++k) {
         const int first = group_offsets[k], last = group_offsets[k + 1];
-        for (int j = first; j < last; ++j) out->member[j] = static_cast<uint8_t>(group_members[j]);
+        for (int j = first; j < last; ++j) {
+            out->member[j] = static_cast<uint8_t>(group_members[j]);
+            out->index_in_group[j] = static_cast<uint8_t>(j - first);
+        }
         out->group_size[last - 1] = static_cast<uint8_t>(last - first);
         out->neg_lr[last - 1] = lrs ? -lrs[k] : -lr;
     }
@@ -107,6 +111,7 @@ bool aligned(const void *p, size_t bytes) { return reinterpret_cast<uintptr_t>(p
 // loads in flight per thread.
 constexpr int kVecBF16 = 8;
 constexpr int kVecF32 = 4;
+constexpr int kVecTree = 4;               // both dtypes, tree summation order (register budget)
 constexpr int kDepthVector = 4;
 constexpr int kDepthScalar = 4;
 constexpr int kVectorBytes = 32;          // base alignment the vector path needs
@@ -149,55 +154,63 @@ extern "C" int star_last_cuda_error(void) { return g_last_cuda_error; }
 
 extern "C" int64_t star_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
-extern "C" star_status_t star_group_update(float *params, float *momentum, const void *const *grads, int W,
-                                           star_dtype_t grad_dtype, int64_t n,
-                                           const int32_t *group_offsets, const int32_t *group_members,
-                                           int n_groups, float lr, float mu, float wd, void *cuda_stream)
+namespace {
+
+// Everything the flat entry points check before a launch.  On STAR_OK either
+// *noop is set (empty tensor or empty schedule: nothing to do) or *args is
+// complete and *vector_ok says whether every buffer allows the vector kernel.
+star_status_t prepare_flat(float *params, float *momentum, const void *const *grads, int W,
+                           star_dtype_t grad_dtype, int64_t n, const int32_t *group_offsets,
+                           const int32_t *group_members, int n_groups, float lr, const float *lrs, float mu,
+                           float wd, FlatArgs *args, bool *vector_ok, bool *noop)
 {
+    *noop = false;
     if (n < 0 || W < 0) return STAR_ERR_INVALID_ARG;
     if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
     if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
-    FlatArgs args;
-    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, lr, &args.sched);
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, lr, &args->sched, lrs);
     if (st != STAR_OK) return st;
-    if (n == 0 || n_groups == 0) return STAR_OK;
+    if (n == 0 || n_groups == 0) {
+        *noop = true;
+        return STAR_OK;
+    }
     if (!params || !momentum || !grads) return STAR_ERR_NULL_POINTER;
-
     const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
     const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
     if (!aligned(params, 4) || !aligned(momentum, 4)) return STAR_ERR_INVALID_ARG;
     if (overlaps(params, state_bytes, momentum, state_bytes)) return STAR_ERR_INVALID_ARG;
-    bool vector_ok = aligned(params, kVectorBytes) && aligned(momentum, kVectorBytes);
-    std::memset(args.grads, 0, sizeof args.grads);
-    for (int j = 0; j < args.sched.n_slots; ++j) {
-        const int w = args.sched.member[j];
+    *vector_ok = aligned(params, kVectorBytes) && aligned(momentum, kVectorBytes);
+    std::memset(args->grads, 0, sizeof args->grads);
+    for (int j = 0; j < args->sched.n_slots; ++j) {
+        const int w = args->sched.member[j];
         const void *g = grads[w];
         if (!g) return STAR_ERR_NULL_POINTER;
         if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
         if (overlaps(g, grad_bytes, params, state_bytes) || overlaps(g, grad_bytes, momentum, state_bytes))
             return STAR_ERR_INVALID_ARG;
-        vector_ok = vector_ok && aligned(g, kVectorBytes);
-        args.grads[w] = g;
+        *vector_ok = *vector_ok && aligned(g, kVectorBytes);
+        args->grads[w] = g;
     }
-    args.params = params;
-    args.momentum = momentum;
-    args.n = n;
-    args.hyper = Hyper{mu, wd};
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    args->params = params;
+    args->momentum = momentum;
+    args->n = n;
+    args->hyper = Hyper{mu, wd};
+    return STAR_OK;
+}
+
+star_status_t dispatch_flat(const FlatArgs &args, star_dtype_t grad_dtype, bool vector_ok, cudaStream_t stream)
+{
     if (grad_dtype == STAR_DTYPE_BF16)
         return vector_ok ? launch_flat<GradBF16, kVecBF16>(args, stream) : launch_flat<GradBF16, 1>(args, stream);
     return vector_ok ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
 }
 
-// Per-group learning rates and parameter snapshots.
-namespace {
-
-template <typename G, int VEC>
+template <typename G, int VEC, bool TREE>
 star_status_t launch_flat_snapshot(const SnapshotArgs &args, cudaStream_t stream)
 {
     static Geometry cache[kMaxDevices];
     constexpr int depth = VEC == 1 ? kDepthScalar : kDepthVector;
-    auto kernel = star_update_flat_snapshot_kernel<G, VEC, depth>;
+    auto kernel = star_update_flat_snapshot_kernel<G, VEC, depth, TREE>;
     int blocks = 0;
     cudaError_t e = resident_blocks(kernel, cache, &blocks);
     if (e != cudaSuccess) return cuda_failed(e);
@@ -212,39 +225,38 @@ star_status_t launch_flat_snapshot(const SnapshotArgs &args, cudaStream_t stream
 
 }  // namespace
 
+extern "C" star_status_t star_group_update(float *params, float *momentum, const void *const *grads, int W,
+                                           star_dtype_t grad_dtype, int64_t n,
+                                           const int32_t *group_offsets, const int32_t *group_members,
+                                           int n_groups, float lr, float mu, float wd, void *cuda_stream)
+{
+    FlatArgs args;
+    bool vector_ok = false, noop = false;
+    const star_status_t st = prepare_flat(params, momentum, grads, W, grad_dtype, n, group_offsets, group_members,
+                                          n_groups, lr, nullptr, mu, wd, &args, &vector_ok, &noop);
+    if (st != STAR_OK || noop) return st;
+    return dispatch_flat(args, grad_dtype, vector_ok, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// Per-group learning rates and parameter snapshots.
 extern "C" star_status_t star_group_update_ex(float *params, float *momentum, const void *const *grads,
                                               int W, star_dtype_t grad_dtype, int64_t n,
                                               const int32_t *group_offsets, const int32_t *group_members,
                                               int n_groups, const float *lrs, float mu, float wd,
-                                              float *const *snapshots, void *cuda_stream)
+                                              float *const *snapshots, star_sum_order_t sum_order,
+                                              void *cuda_stream)
 {
-    if (n < 0 || W < 0) return STAR_ERR_INVALID_ARG;
-    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
-    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    if (sum_order != STAR_SUM_LINEAR && sum_order != STAR_SUM_TREE) return STAR_ERR_INVALID_ARG;
     if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
     SnapshotArgs sargs;
     FlatArgs &args = sargs.flat;
-    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, 0.0f, &args.sched, lrs);
-    if (st != STAR_OK) return st;
-    if (n == 0 || n_groups == 0) return STAR_OK;
-    if (!params || !momentum || !grads) return STAR_ERR_NULL_POINTER;
+    bool vector_ok = false, noop = false;
+    const star_status_t st = prepare_flat(params, momentum, grads, W, grad_dtype, n, group_offsets, group_members,
+                                          n_groups, 0.0f, lrs, mu, wd, &args, &vector_ok, &noop);
+    if (st != STAR_OK || noop) return st;
 
     const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
     const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
-    if (!aligned(params, 4) || !aligned(momentum, 4)) return STAR_ERR_INVALID_ARG;
-    if (overlaps(params, state_bytes, momentum, state_bytes)) return STAR_ERR_INVALID_ARG;
-    bool vector_ok = aligned(params, kVectorBytes) && aligned(momentum, kVectorBytes);
-    std::memset(args.grads, 0, sizeof args.grads);
-    for (int j = 0; j < args.sched.n_slots; ++j) {
-        const int w = args.sched.member[j];
-        const void *g = grads[w];
-        if (!g) return STAR_ERR_NULL_POINTER;
-        if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
-        if (overlaps(g, grad_bytes, params, state_bytes) || overlaps(g, grad_bytes, momentum, state_bytes))
-            return STAR_ERR_INVALID_ARG;
-        vector_ok = vector_ok && aligned(g, kVectorBytes);
-        args.grads[w] = g;
-    }
     std::memset(sargs.snapshots, 0, sizeof sargs.snapshots);
     bool any_snapshot = false;
     for (int k = 0; snapshots && k < n_groups; ++k) {
@@ -261,21 +273,20 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
         sargs.snapshots[group_offsets[k + 1] - 1] = snap;
         any_snapshot = true;
     }
-    args.params = params;
-    args.momentum = momentum;
-    args.n = n;
-    args.hyper = Hyper{mu, wd};
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (!any_snapshot) {                       // per-group rates only: the plain kernel does it
+    if (sum_order == STAR_SUM_TREE) {
         if (grad_dtype == STAR_DTYPE_BF16)
-            return vector_ok ? launch_flat<GradBF16, kVecBF16>(args, stream) : launch_flat<GradBF16, 1>(args, stream);
-        return vector_ok ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
+            return vector_ok ? launch_flat_snapshot<GradBF16, kVecTree, true>(sargs, stream)
+                             : launch_flat_snapshot<GradBF16, 1, true>(sargs, stream);
+        return vector_ok ? launch_flat_snapshot<GradF32, kVecTree, true>(sargs, stream)
+                         : launch_flat_snapshot<GradF32, 1, true>(sargs, stream);
     }
+    if (!any_snapshot) return dispatch_flat(args, grad_dtype, vector_ok, stream);   // per-group rates only
     if (grad_dtype == STAR_DTYPE_BF16)
-        return vector_ok ? launch_flat_snapshot<GradBF16, kVecBF16>(sargs, stream)
-                         : launch_flat_snapshot<GradBF16, 1>(sargs, stream);
-    return vector_ok ? launch_flat_snapshot<GradF32, kVecF32>(sargs, stream)
-                     : launch_flat_snapshot<GradF32, 1>(sargs, stream);
+        return vector_ok ? launch_flat_snapshot<GradBF16, kVecBF16, false>(sargs, stream)
+                         : launch_flat_snapshot<GradBF16, 1, false>(sargs, stream);
+    return vector_ok ? launch_flat_snapshot<GradF32, kVecF32, false>(sargs, stream)
+                     : launch_flat_snapshot<GradF32, 1, false>(sargs, stream);
 }
 
 // ---------------------------------------------------------------------------
@@ -447,7 +458,7 @@ extern "C" star_status_t star_group_update_multi(const star_multi_plan_t *plan,
     if (!plan) return STAR_ERR_NULL_POINTER;
     if (plan->magic != kPlanMagic || !plan->d_workspace) return STAR_ERR_INVALID_ARG;
     MultiArgs args;
-    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, plan->W, lr, &args.sched);
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, plan->W, lr, &args.sched, nullptr);
     if (st != STAR_OK) return st;
     if (plan->n_tiles == 0 || n_groups == 0) return STAR_OK;
     for (int j = 0; j < args.sched.n_slots; ++j)
@@ -539,7 +550,7 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
     if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
     if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
     FlatArgs args;
-    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, lr, &args.sched);
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, lr, &args.sched, nullptr);
     if (st != STAR_OK) return st;
     if (n == 0 || n_groups == 0) return STAR_OK;
     if (!h_params || !h_momentum || !h_grads || !d_workspace) return STAR_ERR_NULL_POINTER;
@@ -615,8 +626,7 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
         args.params = d_p;
         args.momentum = d_v;
         args.n = count;
-        const star_status_t ls = grad_dtype == STAR_DTYPE_BF16 ? launch_flat<GradBF16, kVecBF16>(args, stream)
-                                                               : launch_flat<GradF32, kVecF32>(args, stream);
+        const star_status_t ls = dispatch_flat(args, grad_dtype, true, stream);   // staging buffers are aligned
         if (ls != STAR_OK) return ls;
         e = cudaEventRecord(hp->kernel_done[b], stream);
         if (e != cudaSuccess) return cuda_failed(e);

@@ -34,6 +34,7 @@ struct FlatSchedule {
     int32_t n_slots;
     uint8_t member[kMaxWorkers];       // slot -> worker index
     uint8_t group_size[kMaxWorkers];   // |G_k| on the last slot of group k, else 0
+    uint8_t index_in_group[kMaxWorkers];   // position of the slot inside its group (tree order only)
     float neg_lr[kMaxWorkers];         // -lr_k on the last slot of group k
 };
 
@@ -53,6 +54,7 @@ struct Hyper {
 template <int BYTES> struct Raw;              // BYTES of payload in 32-bit registers
 template <> struct Raw<2>  { uint32_t w[1]; };
 template <> struct Raw<4>  { uint32_t w[1]; };
+template <> struct Raw<8>  { uint32_t w[2]; };
 template <> struct Raw<16> { uint32_t w[4]; };
 template <> struct Raw<32> { uint32_t w[8]; };
 
@@ -70,6 +72,12 @@ template <> __device__ __forceinline__ Raw<4> load_stream<4>(const void *p)
 {
     Raw<4> r;
     asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(r.w[0]) : "l"(p));
+    return r;
+}
+template <> __device__ __forceinline__ Raw<8> load_stream<8>(const void *p)
+{
+    Raw<8> r;
+    asm volatile("ld.global.nc.v2.u32 {%0,%1}, [%2];" : "=r"(r.w[0]), "=r"(r.w[1]) : "l"(p));
     return r;
 }
 template <> __device__ __forceinline__ Raw<16> load_stream<16>(const void *p)
@@ -192,13 +200,26 @@ struct NoSnapshot {
     template <int VEC> __device__ __forceinline__ void operator()(int, int64_t, const float (&)[VEC]) const {}
 };
 
-template <typename G, int VEC, int DEPTH, typename StatePtr, typename GradPtr, typename AfterGroup = NoSnapshot>
+//
+// TREE selects the in-group summation order.  false: left to right.  true:
+// pairwise, as along a binary aggregation tree (Section IV-D2b): the partial
+// sums pending after i leaves are the set bits of i (level l spans 2^l
+// leaves); a new leaf merges with the pending levels below its first clear
+// bit, the group's last leaf with every pending level in ascending order.
+// That is tree(first h) + tree(rest) with h the largest power of two below the
+// group size.  The six pending levels cost 6 * VEC registers, so the tree
+// kernels own 4 elements per thread and are compiled for two resident blocks.
+constexpr int kTreeLevels = 6;             // groups of up to 64 members
+
+template <typename G, int VEC, int DEPTH, bool TREE = false, typename StatePtr, typename GradPtr,
+          typename AfterGroup = NoSnapshot>
 __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first, const FlatSchedule &s,
                                               const Hyper &h, GradPtr grad_ptr,
                                               AfterGroup after_group = AfterGroup())
 {
     constexpr int GB = VEC * G::kBytes;
     float p[VEC], v[VEC], sum[VEC];
+    [[maybe_unused]] float pending[TREE ? kTreeLevels : 1][VEC];
     load_state<VEC>(state_ptr(0) + first, p);
     load_state<VEC>(state_ptr(1) + first, v);
     // -0.0f is the additive identity of IEEE addition (x + -0 == x for every x,
@@ -226,6 +247,37 @@ __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first,
                 if (gs == 1) {                       // singleton group: the mean is the gradient
                     apply_update<VEC>(p, v, f, s.neg_lr[base + j], h);
                     after_group.template operator()<VEC>(base + j, first, p);
+                } else if constexpr (TREE) {
+                    const int leaves_before = s.index_in_group[base + j];
+                    if (gs == 0) {                   // not the last leaf: merge up to the first clear bit
+                        bool stored = false;
+#pragma unroll
+                        for (int l = 0; l < kTreeLevels; ++l) {
+                            if (!stored) {
+                                if (leaves_before >> l & 1) {
+#pragma unroll
+                                    for (int e = 0; e < VEC; ++e) f[e] = __fadd_rn(pending[l][e], f[e]);
+                                } else {
+#pragma unroll
+                                    for (int e = 0; e < VEC; ++e) pending[l][e] = f[e];
+                                    stored = true;
+                                }
+                            }
+                        }
+                    } else {                         // last leaf: fold every pending level
+#pragma unroll
+                        for (int l = 0; l < kTreeLevels; ++l) {
+                            if (leaves_before >> l & 1) {
+#pragma unroll
+                                for (int e = 0; e < VEC; ++e) f[e] = __fadd_rn(pending[l][e], f[e]);
+                            }
+                        }
+                        const float count = static_cast<float>(gs);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) f[e] = __fdiv_rn(f[e], count);
+                        apply_update<VEC>(p, v, f, s.neg_lr[base + j], h);
+                        after_group.template operator()<VEC>(base + j, first, p);
+                    }
                 } else {
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) sum[e] = __fadd_rn(sum[e], f[e]);
@@ -278,9 +330,10 @@ star_update_flat_kernel(const __grid_constant__ FlatArgs a)
     }
 }
 
-// Flat tensor with parameter snapshots: after the update of the group that
-// closes on slot j the parameters are also written to snapshots[j] (if not
-// null) -- the copy the server sends back to that group's workers.
+// Flat tensor with the extended options: parameter snapshots (after the update
+// of the group that closes on slot j the parameters are also written to
+// snapshots[j] if not null -- the copy the server sends back to that group's
+// workers) and the tree summation order.
 struct SnapshotArgs {
     FlatArgs flat;
     float *snapshots[kMaxWorkers];     // indexed by closing slot
@@ -295,8 +348,8 @@ struct StoreSnapshot {
     }
 };
 
-template <typename G, int VEC, int DEPTH>
-__global__ void __launch_bounds__(kBlockThreads, kResidentBlocks)
+template <typename G, int VEC, int DEPTH, bool TREE>
+__global__ void __launch_bounds__(kBlockThreads, TREE ? 2 : kResidentBlocks)
 star_update_flat_snapshot_kernel(const __grid_constant__ SnapshotArgs a)
 {
     const FlatArgs &f = a.flat;
@@ -306,11 +359,11 @@ star_update_flat_snapshot_kernel(const __grid_constant__ SnapshotArgs a)
     auto state_ptr = [&](int which) -> float * { return which == 0 ? f.params : f.momentum; };
     const StoreSnapshot snap{&a};
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kBlockThreads + threadIdx.x; i < n_vec; i += stride)
-        update_vector<G, VEC, DEPTH>(state_ptr, i * VEC, f.sched, f.hyper, grad_ptr, snap);
+        update_vector<G, VEC, DEPTH, TREE>(state_ptr, i * VEC, f.sched, f.hyper, grad_ptr, snap);
     if constexpr (VEC > 1) {
         const int64_t tail = n_vec * VEC + threadIdx.x;
         if (blockIdx.x == 0 && threadIdx.x < VEC && tail < f.n)
-            update_vector<G, 1, DEPTH>(state_ptr, tail, f.sched, f.hyper, grad_ptr, snap);
+            update_vector<G, 1, DEPTH, TREE>(state_ptr, tail, f.sched, f.hyper, grad_ptr, snap);
     }
 }
 

@@ -61,7 +61,27 @@ def fma32(a: Fraction, b: Fraction, c: Fraction) -> Fraction:
     return round_binary32(a * b + c)
 
 
-def grouped_update_exact32(p, v, g, groups, lrs, mu, wd):
+def pairwise_sum32(values):
+    """Pairwise (tree) sum with binary32 rounding, formulated as a binary
+    counter: a new leaf is merged with the pending partial sums of equal span
+    (left operand = the older partial); what is pending at the end is folded
+    from the youngest to the oldest.  For c leaves this builds
+    tree(first h) + tree(rest), h the largest power of two below c."""
+    pending = {}                      # level -> partial sum over 2**level leaves
+    for leaf in values:
+        carry, level = leaf, 0
+        while level in pending:
+            carry = add32(pending.pop(level), carry)
+            level += 1
+        pending[level] = carry
+    levels = sorted(pending)
+    total = pending[levels[0]]
+    for level in levels[1:]:
+        total = add32(pending[level], total)
+    return total
+
+
+def grouped_update_exact32(p, v, g, groups, lrs, mu, wd, tree=False):
     """One element of the grouped update with every step rounded to binary32.
 
     p, v: Fractions; g: list of Fractions per worker; groups: list of lists of
@@ -70,9 +90,12 @@ def grouped_update_exact32(p, v, g, groups, lrs, mu, wd):
     """
     trail = []
     for k, members in enumerate(groups):
-        s = g[members[0]]
-        for w in members[1:]:
-            s = add32(s, g[w])
+        if tree:
+            s = pairwise_sum32([g[w] for w in members])
+        else:
+            s = g[members[0]]
+            for w in members[1:]:
+                s = add32(s, g[w])
         gbar = div32(s, Fraction(len(members)))
         d = fma32(wd, p, gbar)
         v = fma32(mu, v, d)

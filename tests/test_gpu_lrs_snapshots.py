@@ -104,3 +104,45 @@ def test_ex_errors(B):
         B.star_group_update_ex(p, v, grads, [0, 1, 2], [0, 1], [0.1], 0.9, 0.0)
     torch.cuda.synchronize()
     assert torch.equal(p, p0)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_tree_summation_order_matches_oracle(B, dtype):
+    """Group sizes 1..9, 16, 17, 33, 64 in the pairwise (aggregation tree) order."""
+    rng = np.random.default_rng(7)
+    for size in list(range(1, 10)) + [16, 17, 33, 64]:
+        W = min(64, size + 2)
+        for n in (5, 4099, 200_003):
+            p, v, grads = case(n, W, dtype, seed=size * 7 + n)
+            members = [int(w) for w in rng.permutation(W)[:size]]
+            if size >= 3:
+                off, mem = [0, size - 1, size], members
+            else:
+                off, mem = [0, size], members
+            lrs = [0.1] * (len(off) - 1)
+            p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+            g_np = [grad_to_numpy(g) for g in grads]
+            want_snap = [np.zeros(n, np.float32)] + [None] * (len(off) - 2)
+            O.group_update_f32(p_np, v_np, g_np, off, mem, np.array(lrs, np.float32), 0.9, 1e-3,
+                               snapshots=want_snap, sum_order="tree")
+            snap = [torch.empty(n, device="cuda")] + [None] * (len(off) - 2)
+            B.star_group_update_ex(p, v, grads, off, mem, lrs, 0.9, 1e-3, snapshots=snap,
+                                   sum_order=B.STAR_SUM_TREE)
+            torch.cuda.synchronize()
+            assert_matches(p, p_np, "params size=%d n=%d" % (size, n))
+            assert_matches(v, v_np, "momentum size=%d n=%d" % (size, n))
+            assert_matches(snap[0], want_snap[0], "snapshot size=%d n=%d" % (size, n))
+
+
+def test_tree_and_linear_orders_differ_only_in_rounding(B):
+    n = 100_000
+    p, v, grads = case(n, 9, torch.float32, seed=11)
+    q, u = p.clone(), v.clone()
+    off, mem = [0, 9], list(range(9))
+    B.star_group_update_ex(p, v, grads, off, mem, [0.1], 0.9, 1e-4, sum_order=B.STAR_SUM_LINEAR)
+    B.star_group_update_ex(q, u, grads, off, mem, [0.1], 0.9, 1e-4, sum_order=B.STAR_SUM_TREE)
+    torch.cuda.synchronize()
+    assert not torch.equal(p, q)
+    assert float((p - q).abs().max()) <= 8 * 2.0 ** -24 * 0.1
+    with pytest.raises(B.StarError):
+        B.star_group_update_ex(p, v, grads, off, mem, [0.1], 0.9, 1e-4, sum_order=5)

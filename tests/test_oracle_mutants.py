@@ -33,8 +33,11 @@ MUTANTS = {
                                 "for (int k = n_groups - 1; k >= 0; --k) {\n            const int first"),
     "member_index_instead_of_member": ("s = s + grad_at(grads[group_members[j]], grad_dtype, i);",
                                        "s = s + grad_at(grads[j], grad_dtype, i);"),
-    "last_member_skipped": ("for (int j = first + 1; j < last; ++j)\n                s = s + grad_at",
-                            "for (int j = first + 1; j < last - 1; ++j)\n                s = s + grad_at"),
+    "last_member_skipped": ("for (int j = first + 1; j < last; ++j)\n                    s = s + grad_at",
+                            "for (int j = first + 1; j < last - 1; ++j)\n                    s = s + grad_at"),
+    "tree_split_not_a_power_of_two": ("while (2 * h < count)\n        h *= 2;", "h = count / 2;"),
+    "tree_drops_the_right_half": ("tree_sum_f32(grads, dtype, members + h, count - h, i);",
+                                  "tree_sum_f32(grads, dtype, members + h, 1, i);"),
     "bf16_widened_wrongly": ("uint32_t u = (uint32_t)h << 16;", "uint32_t u = (uint32_t)h << 15;"),
     "snapshot_of_the_final_state_only": ("snapshots[k][i] = p;\n        }\n        params[i] = p;",
                                          "snapshots[k][i] = params[i];\n        }\n        params[i] = p;"),
@@ -54,12 +57,12 @@ def build_mutant(tmp_path, name):
     lib = ctypes.CDLL(lib_path)
     common = [ctypes.c_void_p] * 3 + [ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_void_p,
                                       ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
-    lib.oracle_group_update_f32.argtypes = common + [ctypes.c_float, ctypes.c_float, ctypes.c_void_p]
+    lib.oracle_group_update_f32.argtypes = common + [ctypes.c_float, ctypes.c_float, ctypes.c_void_p, ctypes.c_int]
     lib.oracle_group_update_f32.restype = ctypes.c_int
 
-    def update(p, v, grads, off, mem, lrs, mu, wd, snapshots=None):
+    def update(p, v, grads, off, mem, lrs, mu, wd, snapshots=None, sum_order="linear"):
         O._call(lib.oracle_group_update_f32, np.float32, p, v, grads, off, mem, lrs,
-                float(np.float32(mu)), float(np.float32(wd)), snapshots)
+                float(np.float32(mu)), float(np.float32(wd)), snapshots, sum_order)
     return update
 
 
@@ -103,6 +106,19 @@ def pins_accept(update) -> bool:
                     X.to_fraction(np.float32(1e-3)))
                 if X.to_fraction(p[i]) != pe or X.to_fraction(v[i]) != ve:
                     return False
+    # tree order: exact pairwise sums for group sizes 3, 5, 6, 7
+    for size in (3, 5, 6, 7):
+        gs = [rng.normal(0, 0.01, n).astype(np.float32) for _ in range(size)]
+        p, v = p0.copy(), v0.copy()
+        update(p, v, gs, [0, size], list(range(size)), np.float32(0.1), np.float32(0.9), np.float32(1e-3),
+               sum_order="tree")
+        for i in range(n):
+            pe, ve, _ = X.grouped_update_exact32(
+                X.to_fraction(p0[i]), X.to_fraction(v0[i]), [X.to_fraction(g[i]) for g in gs],
+                [list(range(size))], [X.to_fraction(np.float32(0.1))], X.to_fraction(np.float32(0.9)),
+                X.to_fraction(np.float32(1e-3)), tree=True)
+            if X.to_fraction(p[i]) != pe or X.to_fraction(v[i]) != ve:
+                return False
     # PyTorch's SGD, two rounds of three groups (fp32 state: agreement to rounding)
     n = 64
     p0 = rng.normal(0, 0.05, n).astype(np.float32)

@@ -91,6 +91,61 @@ def test_hand_worked_example(variant):
             assert np.all(s == want), name
 
 
+def test_summation_orders_on_the_hand_worked_example():
+    scal, _ = _read_golden()
+    g = [np.full(2, x, np.float32) for x in scal["order_g"]]
+    for order, key in (("linear", "order_linear_p"), ("tree", "order_tree_p")):
+        p, v = np.zeros(2, np.float32), np.zeros(2, np.float32)
+        O.group_update_f32(p, v, g, [0, 4], [0, 1, 2, 3], 1.0, 0.0, 0.0, sum_order=order)
+        assert np.all(p == np.float32(scal[key][0])), order
+    assert scal["order_linear_p"][0] != scal["order_tree_p"][0]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_tree_order_brute_force_against_exact_pairwise_sums(dtype):
+    """Every group size 1..9 (and 16, 17, 33), tree order, exact rounding."""
+    rng = np.random.default_rng(21)
+    n = 4
+    for size in list(range(1, 10)) + [16, 17, 33]:
+        W = size + 1
+        p0 = rng.normal(0, 0.05, n).astype(np.float32)
+        v0 = rng.normal(0, 0.02, n).astype(np.float32)
+        g32 = [(rng.normal(0, 0.01, n) * 10.0 ** rng.integers(-3, 3)).astype(np.float32) for _ in range(W)]
+        grads = [bf16_bits(g) for g in g32] if dtype == "bf16" else g32
+        gval = [bf16_values(b) for b in grads] if dtype == "bf16" else g32
+        members = [int(w) for w in rng.permutation(W)[:size]]
+        groups = [members] if size < 3 else [members[:size - 1], members[size - 1:]]
+        off, mem = csr(groups)
+        p, v = p0.copy(), v0.copy()
+        O.group_update_f32(p, v, grads, off, mem, np.float32(0.1), np.float32(0.9), np.float32(1e-4),
+                           sum_order="tree")
+        for i in range(n):
+            pe, ve, _ = X.grouped_update_exact32(
+                X.to_fraction(p0[i]), X.to_fraction(v0[i]), [X.to_fraction(gv[i]) for gv in gval], groups,
+                [X.to_fraction(np.float32(0.1))] * len(groups), X.to_fraction(np.float32(0.9)),
+                X.to_fraction(np.float32(1e-4)), tree=True)
+            assert X.to_fraction(p[i]) == pe and X.to_fraction(v[i]) == ve, (size, i)
+
+
+def test_tree_and_linear_orders_agree_up_to_rounding_and_exactly_for_small_groups():
+    p0, v0, grads = _random_case(31, 3000, 9, "f32")
+    for size in (1, 2):                      # one or two members: the same operations
+        off, mem = csr([list(range(size))])
+        a, b = p0.copy(), p0.copy()
+        O.group_update_f32(a, v0.copy(), grads, off, mem, 0.1, 0.9, 1e-4, sum_order="linear")
+        O.group_update_f32(b, v0.copy(), grads, off, mem, 0.1, 0.9, 1e-4, sum_order="tree")
+        assert np.array_equal(a, b)
+    off, mem = csr([list(range(9))])
+    P, V = p0.astype(np.float64), v0.astype(np.float64)
+    O.group_update_f64(P, V, grads, off, mem, 0.1, 0.9, 1e-4, sum_order="tree")
+    a, b = p0.copy(), p0.copy()
+    O.group_update_f32(a, v0.copy(), grads, off, mem, 0.1, 0.9, 1e-4, sum_order="linear")
+    O.group_update_f32(b, v0.copy(), grads, off, mem, 0.1, 0.9, 1e-4, sum_order="tree")
+    assert not np.array_equal(a, b)
+    for x in (a, b):
+        assert np.max(np.abs(x - P)) <= 16 * 2.0 ** -24 * 0.2
+
+
 # --------------------------------------------------------------------------
 # 2. exact-rational brute force: every schedule over W<=4, tiny n
 # --------------------------------------------------------------------------
