@@ -1,4 +1,5 @@
 // C-ABI entry points: argument checks on the host, then one kernel launch.
+#include <algorithm>
 #include <atomic>
 #include <cstdint>
 #include <cstring>
@@ -111,7 +112,6 @@ bool aligned(const void *p, size_t bytes) { return reinterpret_cast<uintptr_t>(p
 // loads in flight per thread.
 constexpr int kVecBF16 = 8;
 constexpr int kVecF32 = 4;
-constexpr int kVecTree = 4;               // both dtypes, tree summation order (register budget)
 constexpr int kDepthVector = 4;
 constexpr int kDepthScalar = 4;
 constexpr int kVectorBytes = 32;          // base alignment the vector path needs
@@ -205,7 +205,7 @@ star_status_t dispatch_flat(const FlatArgs &args, star_dtype_t grad_dtype, bool 
     return vector_ok ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
 }
 
-template <typename G, int VEC, bool TREE>
+template <typename G, int VEC, int TREE>
 star_status_t launch_flat_snapshot(const SnapshotArgs &args, cudaStream_t stream)
 {
     static Geometry cache[kMaxDevices];
@@ -221,6 +221,12 @@ star_status_t launch_flat_snapshot(const SnapshotArgs &args, cudaStream_t stream
     if (e != cudaSuccess) return cuda_failed(e);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return STAR_OK;
+}
+
+template <typename G, int VEC, int TREE>
+star_status_t dispatch_snapshot(const SnapshotArgs &args, bool vector_ok, cudaStream_t stream)
+{
+    return vector_ok ? launch_flat_snapshot<G, VEC, TREE>(args, stream) : launch_flat_snapshot<G, 1, TREE>(args, stream);
 }
 
 }  // namespace
@@ -274,19 +280,20 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
         any_snapshot = true;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (sum_order == STAR_SUM_TREE) {
-        if (grad_dtype == STAR_DTYPE_BF16)
-            return vector_ok ? launch_flat_snapshot<GradBF16, kVecTree, true>(sargs, stream)
-                             : launch_flat_snapshot<GradBF16, 1, true>(sargs, stream);
-        return vector_ok ? launch_flat_snapshot<GradF32, kVecTree, true>(sargs, stream)
-                         : launch_flat_snapshot<GradF32, 1, true>(sargs, stream);
+    int largest_group = 1;
+    for (int k = 0; k < n_groups; ++k) largest_group = std::max(largest_group, group_offsets[k + 1] - group_offsets[k]);
+    if (sum_order == STAR_SUM_TREE && largest_group > 2) {      // up to two members both orders are the same sum
+        const bool bf16 = grad_dtype == STAR_DTYPE_BF16;
+        if (largest_group <= 4) return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 2>(sargs, vector_ok, stream)
+                                            : dispatch_snapshot<GradF32, kVecF32, 2>(sargs, vector_ok, stream);
+        if (largest_group <= 16) return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 4>(sargs, vector_ok, stream)
+                                             : dispatch_snapshot<GradF32, kVecF32, 4>(sargs, vector_ok, stream);
+        return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 6>(sargs, vector_ok, stream)
+                    : dispatch_snapshot<GradF32, kVecF32, 6>(sargs, vector_ok, stream);
     }
     if (!any_snapshot) return dispatch_flat(args, grad_dtype, vector_ok, stream);   // per-group rates only
-    if (grad_dtype == STAR_DTYPE_BF16)
-        return vector_ok ? launch_flat_snapshot<GradBF16, kVecBF16, false>(sargs, stream)
-                         : launch_flat_snapshot<GradBF16, 1, false>(sargs, stream);
-    return vector_ok ? launch_flat_snapshot<GradF32, kVecF32, false>(sargs, stream)
-                     : launch_flat_snapshot<GradF32, 1, false>(sargs, stream);
+    return grad_dtype == STAR_DTYPE_BF16 ? dispatch_snapshot<GradBF16, kVecBF16, 0>(sargs, vector_ok, stream)
+                                         : dispatch_snapshot<GradF32, kVecF32, 0>(sargs, vector_ok, stream);
 }
 
 // ---------------------------------------------------------------------------

@@ -207,11 +207,28 @@ struct NoSnapshot {
 // leaves); a new leaf merges with the pending levels below its first clear
 // bit, the group's last leaf with every pending level in ascending order.
 // That is tree(first h) + tree(rest) with h the largest power of two below the
-// group size.  The six pending levels cost 6 * VEC registers, so the tree
-// kernels own 4 elements per thread and are compiled for two resident blocks.
-constexpr int kTreeLevels = 6;             // groups of up to 64 members
+// group size.  A group of c members needs ceil(log2(c)) pending levels of VEC
+// registers each, so the tree kernels are instantiated for 2, 4 and 6 levels
+// (groups of up to 4, 16 and 64 members) and compiled for 3, 2 and 2 resident
+// blocks; TREE is the number of levels, 0 = linear order.
 
-template <typename G, int VEC, int DEPTH, bool TREE = false, typename StatePtr, typename GradPtr,
+// Merge a new leaf with the pending partial sums of levels 0..LEVEL-1 and park
+// the result on LEVEL.
+template <int LEVEL, int VEC, int ROWS>
+__device__ __forceinline__ void tree_merge(float (&pending)[ROWS][VEC], float (&f)[VEC])
+{
+    if constexpr (LEVEL < ROWS) {
+#pragma unroll
+        for (int l = 0; l < LEVEL; ++l) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) f[e] = __fadd_rn(pending[l][e], f[e]);
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) pending[LEVEL][e] = f[e];
+    }
+}
+
+template <typename G, int VEC, int DEPTH, int TREE = 0, typename StatePtr, typename GradPtr,
           typename AfterGroup = NoSnapshot>
 __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first, const FlatSchedule &s,
                                               const Hyper &h, GradPtr grad_ptr,
@@ -219,7 +236,8 @@ __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first,
 {
     constexpr int GB = VEC * G::kBytes;
     float p[VEC], v[VEC], sum[VEC];
-    [[maybe_unused]] float pending[TREE ? kTreeLevels : 1][VEC];
+    constexpr int kTreeLevels = TREE;
+    [[maybe_unused]] float pending[TREE > 0 ? TREE : 1][VEC];
     load_state<VEC>(state_ptr(0) + first, p);
     load_state<VEC>(state_ptr(1) + first, v);
     // -0.0f is the additive identity of IEEE addition (x + -0 == x for every x,
@@ -247,22 +265,18 @@ __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first,
                 if (gs == 1) {                       // singleton group: the mean is the gradient
                     apply_update<VEC>(p, v, f, s.neg_lr[base + j], h);
                     after_group.template operator()<VEC>(base + j, first, p);
-                } else if constexpr (TREE) {
+                } else if constexpr (TREE > 0) {
                     const int leaves_before = s.index_in_group[base + j];
                     if (gs == 0) {                   // not the last leaf: merge up to the first clear bit
-                        bool stored = false;
-#pragma unroll
-                        for (int l = 0; l < kTreeLevels; ++l) {
-                            if (!stored) {
-                                if (leaves_before >> l & 1) {
-#pragma unroll
-                                    for (int e = 0; e < VEC; ++e) f[e] = __fadd_rn(pending[l][e], f[e]);
-                                } else {
-#pragma unroll
-                                    for (int e = 0; e < VEC; ++e) pending[l][e] = f[e];
-                                    stored = true;
-                                }
-                            }
+                        // A real (warp-uniform) branch per level: predicating all six
+                        // levels on every leaf made this path issue-bound.
+                        switch (__ffs(~leaves_before) - 1) {      // number of trailing set bits
+                        case 0: tree_merge<0, VEC>(pending, f); break;
+                        case 1: tree_merge<1, VEC>(pending, f); break;
+                        case 2: tree_merge<2, VEC>(pending, f); break;
+                        case 3: tree_merge<3, VEC>(pending, f); break;
+                        case 4: tree_merge<4, VEC>(pending, f); break;
+                        default: tree_merge<5, VEC>(pending, f); break;
                         }
                     } else {                         // last leaf: fold every pending level
 #pragma unroll
@@ -348,8 +362,13 @@ struct StoreSnapshot {
     }
 };
 
-template <typename G, int VEC, int DEPTH, bool TREE>
-__global__ void __launch_bounds__(kBlockThreads, TREE ? 2 : kResidentBlocks)
+constexpr int tree_resident_blocks(int levels)
+{
+    return levels == 0 ? kResidentBlocks : levels <= 2 ? 3 : 2;
+}
+
+template <typename G, int VEC, int DEPTH, int TREE>
+__global__ void __launch_bounds__(kBlockThreads, tree_resident_blocks(TREE))
 star_update_flat_snapshot_kernel(const __grid_constant__ SnapshotArgs a)
 {
     const FlatArgs &f = a.flat;
