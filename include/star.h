@@ -171,6 +171,29 @@ STAR_API star_status_t star_choose_mode(const double *iter_time, const int32_t *
                                         int32_t *offsets_out, int32_t *members_out,
                                         int *n_groups_out);
 
+/* All-reduce architecture (Section IV-B, Section IV-C1 Eq. 3): remove x of the
+ * stragglers from the ring, attach each to a parent that waits t_w after the
+ * ring's slowest member and adds the gradients of the children that reported
+ * by then.  T_a = (1 + phi / ((W - x + q) M / W)) * (t_ring + t_w).
+ *   iter_time[w]   predicted iteration time in the ring; a worker is a straggler
+ *                  iff (t - min t) / min t > straggler_threshold (Section II: 0.2)
+ *   child_time[w]  predicted iteration time of w when attached to a parent; a
+ *                  removed worker counts (q) iff child_time[w] <= t_ring + t_w
+ *   t_w_max        largest wait considered (t_w in [0, t_w_max])
+ * The x slowest stragglers are removed (x = 0..X, at least one worker stays);
+ * only t_w = 0 and the waits at which one more child makes it are candidates;
+ * ties go to fewer removals, then the shorter wait.  Outputs: *x_out, *t_w_out,
+ * *T_out, removed_out[0..x) (slowest first), and the CSR of the ONE group whose
+ * gradients enter the update (ring members and children in time, ascending
+ * index): on a server holding every worker's buffer the all-reduce mode's
+ * update is star_group_update with that schedule. */
+STAR_API star_status_t star_choose_all_reduce_mode(const double *iter_time, const double *child_time,
+                                                   int W, double phi, double M, double t_w_max,
+                                                   double straggler_threshold, int *x_out,
+                                                   double *t_w_out, double *T_out,
+                                                   int32_t *removed_out, int32_t *offsets_out,
+                                                   int32_t *members_out, int *n_groups_out);
+
 /* Sharding helper (host only).  The path is elementwise, so a job spread over
  * several parameter servers / GPUs (the paper runs one to N PSs per job,
  * Section III set-up) needs no exchange inside it: rank r of world owns the

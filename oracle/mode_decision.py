@@ -96,3 +96,69 @@ def choose_mode(iter_time: Sequence[float], labels: Sequence[int], phi: float,
     if T_d < best_T:
         best_x, best_T = 0, T_d
     return best_x, best_T
+
+
+# ---------------------------------------------------------------------------
+# All-reduce architecture (Section IV-B "All-reduce architecture", Section
+# IV-C1 Eq. 3): remove x of the X stragglers from the ring, attach each to a
+# parent; parents wait t_w after the ring's slowest member is done and add the
+# gradients of the children that have reported by then.
+#
+#   Section II:  d_i = (T_i - min T) / min T;  worker i is a straggler iff d_i > 20 %.
+#   Eq. 3:       T_a = (1 + phi_k / ((N - x + q) M / N)) * (t_ring + t_w)
+#
+# Readings where the paper is silent or loose:
+#   * which x stragglers are removed: the x slowest (ties: larger index first).
+#   * "q = removed stragglers with new iteration times no higher than t_w": a
+#     removed worker w has a predicted iteration time as a child, child_time[w];
+#     it counts iff child_time[w] <= t_ring + t_w, i.e. its report is in before
+#     its parent stops waiting.
+#   * range of t_w: 0 <= t_w <= t_w_max.  Only t_w = 0 and the values at which
+#     one more child makes it, child_time[w] - t_ring, can be optimal.
+#   * ties: fewer removed workers, then the shorter wait.
+# The gradients that enter the update are those of the ring members and of the
+# q children in time: on a parameter server holding all buffers this is ONE
+# group of N - x + q workers (a partial cover of the N workers).
+# ---------------------------------------------------------------------------
+def deviation_ratios(iter_time: Sequence[float]) -> List[float]:
+    fastest = min(iter_time)
+    return [(t - fastest) / fastest for t in iter_time]
+
+
+def stragglers(iter_time: Sequence[float], threshold: float = 0.2) -> List[int]:
+    return [w for w, d in enumerate(deviation_ratios(iter_time)) if d > threshold]
+
+
+def time_all_reduce(iter_time: Sequence[float], child_time: Sequence[float], removed: Sequence[int],
+                    t_w: float, phi: float, M: float) -> Tuple[float, List[int]]:
+    """Eq. 3 for a given set of removed workers and wait time.  Returns (T_a,
+    the removed workers whose gradients still arrive in time)."""
+    N = len(iter_time)
+    ring = [w for w in range(N) if w not in removed]
+    t_ring = max(iter_time[w] for w in ring)
+    in_time = [w for w in removed if child_time[w] <= t_ring + t_w]
+    x, q = len(removed), len(in_time)
+    return (1.0 + phi / ((N - x + q) * M / N)) * (t_ring + t_w), in_time
+
+
+def choose_all_reduce_mode(iter_time: Sequence[float], child_time: Sequence[float], phi: float, M: float,
+                           t_w_max: float, threshold: float = 0.2):
+    """Enumerate x = 0..X and the candidate waits; returns
+    (x, t_w, T_a, removed workers, contributing workers sorted ascending)."""
+    N = len(iter_time)
+    slow_first = sorted(stragglers(iter_time, threshold), key=lambda w: (-iter_time[w], -w))
+    best = None
+    for x in range(0, min(len(slow_first), N - 1) + 1):
+        removed = slow_first[:x]
+        ring = [w for w in range(N) if w not in removed]
+        t_ring = max(iter_time[w] for w in ring)
+        waits = {0.0}
+        for w in removed:
+            need = child_time[w] - t_ring
+            if 0.0 < need <= t_w_max:
+                waits.add(need)
+        for t_w in sorted(waits):
+            T, in_time = time_all_reduce(iter_time, child_time, removed, t_w, phi, M)
+            if best is None or T < best[2]:
+                best = (x, t_w, T, list(removed), sorted(ring + in_time))
+    return best

@@ -92,6 +92,8 @@ def _load() -> ctypes.CDLL:
     lib.star_choose_mode.argtypes = [c_vp, c_vp, c_int, ctypes.c_double, ctypes.c_double, c_vp, c_vp,
                                      c_vp, c_vp, c_vp]
     lib.star_choose_mode.restype = c_int
+    lib.star_choose_all_reduce_mode.argtypes = [c_vp, c_vp, c_int] + [ctypes.c_double] * 4 + [c_vp] * 7
+    lib.star_choose_all_reduce_mode.restype = c_int
     lib.star_shard_range.argtypes = [c_i64, c_int, c_int, c_i64, c_vp, c_vp]
     lib.star_shard_range.restype = c_int
     lib.star_host_workspace_bytes.argtypes = [c_int, c_int, c_i64, c_vp]
@@ -219,6 +221,21 @@ def star_choose_mode(iter_time: Sequence[float], cluster_of_worker: Optional[Seq
     _check(_lib.star_choose_mode(_f64(iter_time), clusters, W, phi, M, ctypes.byref(x), ctypes.byref(T),
                                  offsets, members, ctypes.byref(K)), "star_choose_mode")
     return x.value, T.value, _unpack(offsets, members, K)
+
+
+def star_choose_all_reduce_mode(iter_time: Sequence[float], child_time: Sequence[float], phi: float,
+                                M: float, t_w_max: float, straggler_threshold: float = 0.2):
+    """(x, t_w, T_a, removed workers, schedule of the one contributing group)."""
+    W = len(iter_time)
+    if len(child_time) != W:
+        raise StarError(STAR_ERR_INVALID_ARG, "star_choose_all_reduce_mode")
+    x, t_w, T, K = ctypes.c_int(0), ctypes.c_double(0.0), ctypes.c_double(0.0), ctypes.c_int(0)
+    removed, offsets, members = _i32([0] * W), _i32([0] * (W + 1)), _i32([0] * W)
+    _check(_lib.star_choose_all_reduce_mode(_f64(iter_time), _f64(child_time), W, phi, M, t_w_max,
+                                            straggler_threshold, ctypes.byref(x), ctypes.byref(t_w),
+                                            ctypes.byref(T), removed, offsets, members, ctypes.byref(K)),
+           "star_choose_all_reduce_mode")
+    return x.value, t_w.value, T.value, list(removed[: x.value]), _unpack(offsets, members, K)
 
 
 def star_shard_range(n: int, world: int, rank: int, align: int = 16) -> Tuple[int, int]:

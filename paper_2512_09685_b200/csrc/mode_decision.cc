@@ -134,3 +134,85 @@ extern "C" star_status_t star_choose_mode(const double *iter_time, const int32_t
     std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return iter_time[a] < iter_time[b]; });
     return star_schedule_static_x(order.data(), W, W, best_x, 1, offsets_out, members_out, n_groups_out);
 }
+
+// ---------------------------------------------------------------------------
+// All-reduce architecture: which stragglers leave the ring and how long the
+// parents wait (Section IV-C1, Eq. 3).
+// ---------------------------------------------------------------------------
+extern "C" star_status_t star_choose_all_reduce_mode(const double *iter_time, const double *child_time, int W,
+                                                     double phi, double M, double t_w_max,
+                                                     double straggler_threshold, int *x_out, double *t_w_out,
+                                                     double *T_out, int32_t *removed_out, int32_t *offsets_out,
+                                                     int32_t *members_out, int *n_groups_out)
+{
+    if (!iter_time || !child_time || !x_out || !t_w_out || !T_out || !removed_out || !offsets_out || !members_out ||
+        !n_groups_out)
+        return STAR_ERR_NULL_POINTER;
+    if (W < 1 || !(phi >= 0.0) || !(M > 0.0) || !(t_w_max >= 0.0) || !(straggler_threshold >= 0.0) ||
+        !std::isfinite(phi) || !std::isfinite(M) || !std::isfinite(t_w_max))
+        return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    if (!times_ok(iter_time, W) || !times_ok(child_time, W)) return STAR_ERR_INVALID_ARG;
+    const double N = static_cast<double>(W);
+
+    // Stragglers (Section II: deviation ratio above the threshold), slowest first.
+    const double fastest = *std::min_element(iter_time, iter_time + W);
+    std::vector<int32_t> slow;
+    for (int w = 0; w < W; ++w)
+        if ((iter_time[w] - fastest) / fastest > straggler_threshold) slow.push_back(w);
+    std::sort(slow.begin(), slow.end(), [&](int32_t a, int32_t b) {
+        if (iter_time[a] != iter_time[b]) return iter_time[a] > iter_time[b];
+        return a > b;
+    });
+
+    bool have = false;
+    int best_x = 0;
+    double best_wait = 0.0, best_T = 0.0;
+    const int max_removed = std::min<int>(static_cast<int>(slow.size()), W - 1);
+    for (int x = 0; x <= max_removed; ++x) {
+        std::vector<bool> is_removed(W, false);
+        for (int j = 0; j < x; ++j) is_removed[slow[j]] = true;
+        double t_ring = 0.0;
+        for (int w = 0; w < W; ++w)
+            if (!is_removed[w]) t_ring = std::max(t_ring, iter_time[w]);
+        // Only t_w = 0 and the waits at which one more child makes it can be optimal.
+        std::vector<double> waits{0.0};
+        for (int j = 0; j < x; ++j) {
+            const double need = child_time[slow[j]] - t_ring;
+            if (need > 0.0 && need <= t_w_max) waits.push_back(need);
+        }
+        std::sort(waits.begin(), waits.end());
+        waits.erase(std::unique(waits.begin(), waits.end()), waits.end());
+        for (double t_w : waits) {
+            int q = 0;
+            for (int j = 0; j < x; ++j)
+                if (child_time[slow[j]] <= t_ring + t_w) ++q;
+            const double T = (1.0 + phi / (static_cast<double>(W - x + q) * M / N)) * (t_ring + t_w);
+            if (!have || T < best_T) {          // strict: ties keep fewer removals, then the shorter wait
+                have = true;
+                best_x = x;
+                best_wait = t_w;
+                best_T = T;
+            }
+        }
+    }
+    *x_out = best_x;
+    *t_w_out = best_wait;
+    *T_out = best_T;
+    std::vector<bool> is_removed(W, false);
+    for (int j = 0; j < best_x; ++j) {
+        removed_out[j] = slow[j];
+        is_removed[slow[j]] = true;
+    }
+    double t_ring = 0.0;
+    for (int w = 0; w < W; ++w)
+        if (!is_removed[w]) t_ring = std::max(t_ring, iter_time[w]);
+    // One group: the ring members and the children whose reports are in on time.
+    int32_t count = 0;
+    for (int w = 0; w < W; ++w)
+        if (!is_removed[w] || child_time[w] <= t_ring + best_wait) members_out[count++] = w;
+    offsets_out[0] = 0;
+    offsets_out[1] = count;
+    *n_groups_out = 1;
+    return STAR_OK;
+}

@@ -74,3 +74,36 @@ def test_mode_decision_rejects_bad_input():
         B.star_mode_times([1.0, 2.0], [0, -1], 1.0, 64.0)
     with pytest.raises(B.StarError):
         B.star_choose_mode([], None, 1.0, 64.0)
+
+
+def test_all_reduce_mode_matches_oracle():
+    rng = random.Random(4)
+    seen_x = set()
+    for _ in range(400):
+        W = rng.randint(1, 12)
+        t = [rng.uniform(0.1, 0.3) * rng.choice([1, 1, 1, 2, 6]) for _ in range(W)]
+        child = [ti * rng.uniform(0.3, 1.0) for ti in t]
+        phi, M, t_w_max = rng.choice([0.0, 5.0, 200.0, 1e5]), 512.0, rng.choice([0.0, 0.05, 0.5])
+        x, t_w, T, removed, (off, mem) = B.star_choose_all_reduce_mode(t, child, phi, M, t_w_max)
+        wx, wt, wT, wremoved, wused = D.choose_all_reduce_mode(t, child, phi, M, t_w_max)
+        assert (x, removed, mem) == (wx, wremoved, wused) and off == [0, len(wused)]
+        assert t_w == pytest.approx(wt, abs=1e-15) and T == pytest.approx(wT, rel=1e-14)
+        assert B.star_schedule_validate(off, mem, 1, W) == B.STAR_OK
+        seen_x.add(x)
+    assert {0, 1, 2} <= seen_x
+
+
+def test_all_reduce_worked_example_through_the_library():
+    x, t_w, T, removed, sched = B.star_choose_all_reduce_mode([1.0, 1.0, 2.0, 4.0], [9.0, 9.0, 1.5, 3.0],
+                                                              64.0, 128.0, 1.0)
+    assert (x, t_w, removed, sched) == (2, 0.0, [3, 2], ([0, 2], [0, 1])) and T == pytest.approx(2.0)
+    # children that are quick once attached and a noisy gradient (large phi): waiting for them pays,
+    # (1 + phi/128) * 1.2 < (1 + phi/64) * 1
+    x, t_w, T, removed, sched = B.star_choose_all_reduce_mode([1.0, 1.0, 2.0, 4.0], [9.0, 9.0, 1.1, 1.2],
+                                                              1e4, 128.0, 1.0)
+    assert (x, removed, sched) == (2, [3, 2], ([0, 4], [0, 1, 2, 3]))
+    assert t_w == pytest.approx(0.2) and T == pytest.approx((1 + 1e4 / 128) * 1.2)
+    with pytest.raises(B.StarError):
+        B.star_choose_all_reduce_mode([1.0, 2.0], [1.0], 1.0, 64.0, 0.1)
+    with pytest.raises(B.StarError):
+        B.star_choose_all_reduce_mode([1.0, 2.0], [1.0, -2.0], 1.0, 64.0, 0.1)

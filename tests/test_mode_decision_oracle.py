@@ -86,3 +86,46 @@ def test_clustering_matches_scipy_average_linkage(seed):
     for thr in (0.05, 0.3, 1.5):
         want = canonical(fcluster(Z, thr, criterion="distance"))
         assert D.agglomerative_clusters(list(t), max_distance=thr) == want
+
+
+# --------------------------------------------------------------------------
+# all-reduce architecture, Eq. 3
+# --------------------------------------------------------------------------
+def test_straggler_rule_of_section_ii():
+    assert D.deviation_ratios([1.0, 1.2, 1.21, 2.0]) == pytest.approx([0.0, 0.2, 0.21, 1.0])
+    assert D.stragglers([1.0, 1.2, 1.21, 2.0]) == [2, 3]          # strictly more than 20 %
+
+
+def test_all_reduce_hand_worked_example():
+    g = read_golden()
+    t, M, phi = g["t"], g["M"][0], g["phi"][0]
+    child, t_w_max = g["ar_child_time"], g["ar_t_w_max"][0]
+    assert D.time_all_reduce(t, child, [], 0.0, phi, M)[0] == pytest.approx(6.0)
+    assert D.time_all_reduce(t, child, [3], 0.0, phi, M) == (pytest.approx(10 / 3), [])
+    assert D.time_all_reduce(t, child, [3], 1.0, phi, M) == (pytest.approx(4.5), [3])
+    assert D.time_all_reduce(t, child, [3, 2], 0.5, phi, M) == (pytest.approx(2.5), [2])
+    x, t_w, T, removed, used = D.choose_all_reduce_mode(t, child, phi, M, t_w_max)
+    assert (x, t_w, removed, used) == (int(g["ar_best_x"][0]), g["ar_best_t_w"][0], [3, 2], [0, 1])
+    assert T == pytest.approx(g["ar_best_T"][0])
+
+
+def test_eq3_without_removal_is_ssgd_eq1():
+    t = [0.3, 0.5, 0.25, 0.9]
+    T, used = D.time_all_reduce(t, t, [], 0.0, 12.0, 256.0)
+    assert T == pytest.approx(D.time_static_x(t, 4, 12.0, 256.0)) and used == []
+
+
+def test_breakpoint_enumeration_equals_a_dense_scan_of_wait_times():
+    rng = np.random.default_rng(3)
+    for _ in range(100):
+        N = int(rng.integers(2, 9))
+        t = list(rng.uniform(0.1, 0.3, N) * rng.choice([1, 1, 2, 5], N))
+        child = [ti * rng.uniform(0.3, 1.0) for ti in t]
+        phi, M, t_w_max = float(rng.choice([1.0, 50.0, 5000.0])), 512.0, 0.2
+        x, t_w, T, removed, used = D.choose_all_reduce_mode(t, child, phi, M, t_w_max)
+        slow = sorted(D.stragglers(t), key=lambda w: (-t[w], -w))
+        dense = min(D.time_all_reduce(t, child, slow[:xx], tw, phi, M)[0]
+                    for xx in range(0, min(len(slow), N - 1) + 1) for tw in np.linspace(0, t_w_max, 401))
+        assert T <= dense * (1 + 1e-12)
+        assert T == pytest.approx(D.time_all_reduce(t, child, removed, t_w, phi, M)[0])
+        assert sorted(set(range(N)) - set(removed)) == [w for w in used if w not in removed]
