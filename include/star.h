@@ -40,7 +40,7 @@
  *   - There is no CPU path: without a usable CUDA device the compute entry
  *     points return STAR_ERR_CUDA.
  *   - params, momentum and the scheduled gradient buffers must not overlap.
- *     Element-size alignment is required (4 bytes fp32, 2 bytes bf16); 16-byte
+ *     Element-size alignment is required (4 bytes fp32, 2 bytes bf16); 32-byte
  *     aligned buffers take the vector path, others a slower scalar path with
  *     identical results.
  */

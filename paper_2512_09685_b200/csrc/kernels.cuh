@@ -324,7 +324,7 @@ struct FlatArgs {
     Hyper hyper;
 };
 
-// Vector kernel: requires 16-byte (VEC*kBytes == 16) or 32-byte aligned bases.
+// Vector kernel: requires 32-byte aligned bases (p and v move in 32-byte accesses when VEC = 8).
 // Grid-stride over vectors; the last < VEC elements are done one by one by the
 // first threads of block 0.
 template <typename G, int VEC, int DEPTH>
