@@ -107,17 +107,25 @@ class ClockSampler:
         except Exception:
             self.nv = None
 
-    def _loop(self):
+    def sample(self):
+        """One reading, now (also called from the timing loop right after the last
+        launch is queued, so that even a very short region has a sample taken
+        while the GPU is busy)."""
         nv = self.nv
+        if nv is None:
+            return
+        try:
+            self.sm.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+            mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+            for name, bit in self.REASONS:
+                if mask & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _loop(self):
         while not self._stop.is_set():
-            try:
-                self.sm.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
-                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
-                for name, bit in self.REASONS:
-                    if mask & bit:
-                        self.reasons.add(name)
-            except Exception:
-                pass
+            self.sample()
             self._stop.wait(self.period)
 
     def __enter__(self):
@@ -222,6 +230,8 @@ def time_device(dw: DeviceWorkload, steps: int, warmup: int, dist, sampler=None)
     for i in range(steps):
         scheduled += dw.step()
     end.record()
+    if sampler is not None:
+        sampler.sample()
     torch.cuda.synchronize()
     if sampler is not None:
         sampler.__exit__(None, None, None)

@@ -40,9 +40,10 @@
  *   - There is no CPU path: without a usable CUDA device the compute entry
  *     points return STAR_ERR_CUDA.
  *   - params, momentum and the scheduled gradient buffers must not overlap.
- *     Element-size alignment is required (4 bytes fp32, 2 bytes bf16); 32-byte
- *     aligned buffers take the vector path, others a slower scalar path with
- *     identical results.
+ *     Element-size alignment is required (4 bytes fp32, 2 bytes bf16).  Buffers
+ *     aligned to 32 bytes take the full-width vector path; less aligned
+ *     buffers take a narrower or element-by-element path with identical
+ *     results (slower).
  */
 #ifndef STAR_H_
 #define STAR_H_

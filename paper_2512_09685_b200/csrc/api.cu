@@ -114,7 +114,35 @@ constexpr int kVecBF16 = 8;
 constexpr int kVecF32 = 4;
 constexpr int kDepthVector = 4;
 constexpr int kDepthScalar = 4;
-constexpr int kVectorBytes = 32;          // base alignment the vector path needs
+constexpr int kVecBF16Half = 4;           // bf16 with buffers aligned for 16-byte state / 8-byte gradient accesses
+
+// Alignment of the buffers of a call: the smallest power of two (capped at 32)
+// that divides every state (p, v, snapshot) address, and every gradient address.
+struct Alignment {
+    unsigned state = 32, grad = 32;
+    static unsigned of(const void *p)
+    {
+        const uintptr_t a = reinterpret_cast<uintptr_t>(p);
+        unsigned k = 32;
+        while (k > 1 && a % k != 0) k /= 2;
+        return k;
+    }
+    void add_state(const void *p) { state = std::min(state, of(p)); }
+    void add_grad(const void *p) { grad = std::min(grad, of(p)); }
+};
+
+// Elements per thread the alignment allows.  bf16: 8 (32-byte state accesses,
+// 16-byte gradient loads) or 4 (16 / 8 bytes); fp32: 4 (16-byte accesses); else
+// the element-by-element kernel.
+int vector_width(star_dtype_t dt, const Alignment &al)
+{
+    if (dt == STAR_DTYPE_BF16) {
+        if (al.state >= 32 && al.grad >= 16) return kVecBF16;
+        if (al.state >= 16 && al.grad >= 8) return kVecBF16Half;
+        return 1;
+    }
+    return al.state >= 16 && al.grad >= 16 ? kVecF32 : 1;
+}
 
 template <typename G, int VEC>
 star_status_t launch_flat(const FlatArgs &args, cudaStream_t stream)
@@ -158,11 +186,11 @@ namespace {
 
 // Everything the flat entry points check before a launch.  On STAR_OK either
 // *noop is set (empty tensor or empty schedule: nothing to do) or *args is
-// complete and *vector_ok says whether every buffer allows the vector kernel.
+// complete and *align holds the alignment of its buffers.
 star_status_t prepare_flat(float *params, float *momentum, const void *const *grads, int W,
                            star_dtype_t grad_dtype, int64_t n, const int32_t *group_offsets,
                            const int32_t *group_members, int n_groups, float lr, const float *lrs, float mu,
-                           float wd, FlatArgs *args, bool *vector_ok, bool *noop)
+                           float wd, FlatArgs *args, Alignment *align, bool *noop)
 {
     *noop = false;
     if (n < 0 || W < 0) return STAR_ERR_INVALID_ARG;
@@ -179,7 +207,8 @@ star_status_t prepare_flat(float *params, float *momentum, const void *const *gr
     const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
     if (!aligned(params, 4) || !aligned(momentum, 4)) return STAR_ERR_INVALID_ARG;
     if (overlaps(params, state_bytes, momentum, state_bytes)) return STAR_ERR_INVALID_ARG;
-    *vector_ok = aligned(params, kVectorBytes) && aligned(momentum, kVectorBytes);
+    align->add_state(params);
+    align->add_state(momentum);
     std::memset(args->grads, 0, sizeof args->grads);
     for (int j = 0; j < args->sched.n_slots; ++j) {
         const int w = args->sched.member[j];
@@ -188,7 +217,7 @@ star_status_t prepare_flat(float *params, float *momentum, const void *const *gr
         if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
         if (overlaps(g, grad_bytes, params, state_bytes) || overlaps(g, grad_bytes, momentum, state_bytes))
             return STAR_ERR_INVALID_ARG;
-        *vector_ok = *vector_ok && aligned(g, kVectorBytes);
+        align->add_grad(g);
         args->grads[w] = g;
     }
     args->params = params;
@@ -198,11 +227,16 @@ star_status_t prepare_flat(float *params, float *momentum, const void *const *gr
     return STAR_OK;
 }
 
-star_status_t dispatch_flat(const FlatArgs &args, star_dtype_t grad_dtype, bool vector_ok, cudaStream_t stream)
+star_status_t dispatch_flat(const FlatArgs &args, star_dtype_t grad_dtype, const Alignment &align,
+                            cudaStream_t stream)
 {
-    if (grad_dtype == STAR_DTYPE_BF16)
-        return vector_ok ? launch_flat<GradBF16, kVecBF16>(args, stream) : launch_flat<GradBF16, 1>(args, stream);
-    return vector_ok ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
+    const int vec = vector_width(grad_dtype, align);
+    if (grad_dtype == STAR_DTYPE_BF16) {
+        if (vec == kVecBF16) return launch_flat<GradBF16, kVecBF16>(args, stream);
+        if (vec == kVecBF16Half) return launch_flat<GradBF16, kVecBF16Half>(args, stream);
+        return launch_flat<GradBF16, 1>(args, stream);
+    }
+    return vec == kVecF32 ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
 }
 
 template <typename G, int VEC, int TREE>
@@ -223,6 +257,7 @@ star_status_t launch_flat_snapshot(const SnapshotArgs &args, cudaStream_t stream
     return STAR_OK;
 }
 
+// The extended kernels come in the full vector width and element by element only.
 template <typename G, int VEC, int TREE>
 star_status_t dispatch_snapshot(const SnapshotArgs &args, bool vector_ok, cudaStream_t stream)
 {
@@ -237,11 +272,12 @@ extern "C" star_status_t star_group_update(float *params, float *momentum, const
                                            int n_groups, float lr, float mu, float wd, void *cuda_stream)
 {
     FlatArgs args;
-    bool vector_ok = false, noop = false;
+    Alignment align;
+    bool noop = false;
     const star_status_t st = prepare_flat(params, momentum, grads, W, grad_dtype, n, group_offsets, group_members,
-                                          n_groups, lr, nullptr, mu, wd, &args, &vector_ok, &noop);
+                                          n_groups, lr, nullptr, mu, wd, &args, &align, &noop);
     if (st != STAR_OK || noop) return st;
-    return dispatch_flat(args, grad_dtype, vector_ok, static_cast<cudaStream_t>(cuda_stream));
+    return dispatch_flat(args, grad_dtype, align, static_cast<cudaStream_t>(cuda_stream));
 }
 
 // Per-group learning rates and parameter snapshots.
@@ -256,9 +292,10 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
     if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
     SnapshotArgs sargs;
     FlatArgs &args = sargs.flat;
-    bool vector_ok = false, noop = false;
+    Alignment align;
+    bool noop = false;
     const star_status_t st = prepare_flat(params, momentum, grads, W, grad_dtype, n, group_offsets, group_members,
-                                          n_groups, 0.0f, lrs, mu, wd, &args, &vector_ok, &noop);
+                                          n_groups, 0.0f, lrs, mu, wd, &args, &align, &noop);
     if (st != STAR_OK || noop) return st;
 
     const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
@@ -275,11 +312,12 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
             if (overlaps(snap, state_bytes, args.grads[args.sched.member[j]], grad_bytes)) return STAR_ERR_INVALID_ARG;
         for (int l = 0; l < k; ++l)
             if (snapshots[l] && overlaps(snap, state_bytes, snapshots[l], state_bytes)) return STAR_ERR_INVALID_ARG;
-        vector_ok = vector_ok && aligned(snap, kVectorBytes);
+        align.add_state(snap);
         sargs.snapshots[group_offsets[k + 1] - 1] = snap;
         any_snapshot = true;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool vector_ok = vector_width(grad_dtype, align) == (grad_dtype == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32);
     int largest_group = 1;
     for (int k = 0; k < n_groups; ++k) largest_group = std::max(largest_group, group_offsets[k + 1] - group_offsets[k]);
     if (sum_order == STAR_SUM_TREE && largest_group > 2) {      // up to two members both orders are the same sum
@@ -291,7 +329,7 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
         return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 6>(sargs, vector_ok, stream)
                     : dispatch_snapshot<GradF32, kVecF32, 6>(sargs, vector_ok, stream);
     }
-    if (!any_snapshot) return dispatch_flat(args, grad_dtype, vector_ok, stream);   // per-group rates only
+    if (!any_snapshot) return dispatch_flat(args, grad_dtype, align, stream);   // per-group rates only
     return grad_dtype == STAR_DTYPE_BF16 ? dispatch_snapshot<GradBF16, kVecBF16, 0>(sargs, vector_ok, stream)
                                          : dispatch_snapshot<GradF32, kVecF32, 0>(sargs, vector_ok, stream);
 }
@@ -413,13 +451,14 @@ extern "C" star_status_t star_multi_prepare(int n_tensors, float *const *params,
         e.size = size;
         e.first_tile = next_tile;
         e.pad = 0;
-        bool vector_ok = true;
+        Alignment align;
         if (size > 0) {
             if (!params[t] || !momentum[t]) return STAR_ERR_NULL_POINTER;
             if (!aligned(params[t], 4) || !aligned(momentum[t], 4)) return STAR_ERR_INVALID_ARG;
             const size_t state_bytes = static_cast<size_t>(size) * 4;
             if (overlaps(params[t], state_bytes, momentum[t], state_bytes)) return STAR_ERR_INVALID_ARG;
-            vector_ok = aligned(params[t], kVectorBytes) && aligned(momentum[t], kVectorBytes);
+            align.add_state(params[t]);
+            align.add_state(momentum[t]);
         }
         for (int w = 0; w < W; ++w) {
             const void *g = grads[static_cast<size_t>(t) * W + w];
@@ -433,9 +472,9 @@ extern "C" star_status_t star_multi_prepare(int n_tensors, float *const *params,
             const size_t state_bytes = static_cast<size_t>(size) * 4, grad_bytes = static_cast<size_t>(size) * gsize;
             if (overlaps(g, grad_bytes, params[t], state_bytes) || overlaps(g, grad_bytes, momentum[t], state_bytes))
                 return STAR_ERR_INVALID_ARG;
-            vector_ok = vector_ok && aligned(g, kVectorBytes);
+            align.add_grad(g);
         }
-        e.vector_ok = vector_ok ? 1 : 0;
+        e.vec = vector_width(grad_dtype, align);
         const int64_t tiles_here = (size + tile - 1) / tile;
         for (int64_t i = 0; i < tiles_here; ++i) tile_tensor[next_tile + i] = t;
         next_tile += tiles_here;
@@ -633,7 +672,7 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
         args.params = d_p;
         args.momentum = d_v;
         args.n = count;
-        const star_status_t ls = dispatch_flat(args, grad_dtype, true, stream);   // staging buffers are aligned
+        const star_status_t ls = dispatch_flat(args, grad_dtype, Alignment{}, stream);   // staging buffers are aligned
         if (ls != STAR_OK) return ls;
         e = cudaEventRecord(hp->kernel_done[b], stream);
         if (e != cudaSuccess) return cuda_failed(e);

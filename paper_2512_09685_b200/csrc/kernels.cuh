@@ -397,7 +397,7 @@ struct TensorEntry {
     float *momentum;
     int64_t size;          // elements
     int64_t first_tile;
-    int32_t vector_ok;     // all of the tensor's buffers are aligned for the vector path
+    int32_t vec;           // elements per thread the tensor's buffer alignment allows (full width or less)
     int32_t pad;
 };
 
@@ -412,8 +412,9 @@ struct MultiArgs {
 };
 
 // Element-by-element path for the ragged end of a tensor and for tensors whose
-// buffers are not aligned for vector access.  Kept out of line: it is cold, and
-// inlining it next to the vector path costs registers there.
+// buffers are not aligned for the full vector width.  Kept out of line: it is
+// cold, and inlining it next to the vector path costs registers there.
+// Handles elements first, first + step, ... below end.
 template <typename G, int DEPTH>
 __device__ __noinline__ void update_elements(const TensorEntry &te, const unsigned long long *row,
                                              int64_t first, int64_t end, int64_t step,
@@ -441,7 +442,7 @@ star_update_multi_kernel(const __grid_constant__ MultiArgs a)
             reinterpret_cast<const unsigned long long *>(a.grads) + static_cast<int64_t>(t) * a.W;
         const int64_t begin = (tile - te.first_tile) * kTile;
         const int64_t size = te.size;
-        if (te.vector_ok) {
+        if (te.vec == VEC) {
             const int64_t i = begin + static_cast<int64_t>(threadIdx.x) * VEC;
             if (i + VEC <= size) {
                 auto grad_ptr = [&](int slot) -> const void * {
@@ -460,6 +461,9 @@ star_update_multi_kernel(const __grid_constant__ MultiArgs a)
                 update_elements<G, DEPTH>(te, row, i, size, 1, a.sched, a.hyper);
             }
         } else {
+            // Not aligned for the full vector width: element by element.  (A
+            // narrower vector path here was measured to cost the aligned path
+            // a third of its bandwidth through register spills.)
             const int64_t end = min(size, begin + kTile);
             update_elements<G, DEPTH>(te, row, begin + threadIdx.x, end, kBlockThreads, a.sched, a.hyper);
         }
