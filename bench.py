@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # workload, with the SHA-256 of the kernel sources the capture was taken on:
 # once the sources differ the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "cfg1_resnet50": (787.8e6, "4ece91ef8e81660e9df4dbf35e9dc8e2e795a8cf298fcc4410c9200da8371dbc"),
+    "cfg1_resnet50": (787.9e6, "f4cb3bae04c5d294af704d9dd8d6983a27d34285951ce88919069037b6c17f2c"),
 }
 
 
