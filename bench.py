@@ -256,6 +256,30 @@ def time_device(dw: DeviceWorkload, steps: int, warmup: int, dist, sampler=None)
     return seconds, per_launch, nbytes, launches
 
 
+def time_graph_replay(dw: DeviceWorkload, rounds: int, replays: int) -> float:
+    """ms per round when `rounds` rounds are captured once in a CUDA graph and
+    replayed `replays` times."""
+    torch = dw.torch
+    dw.step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(rounds):
+                dw.step()
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (rounds * replays)
+
+
 def time_e2e(w, steps: int, warmup: int, dist):
     """The same rounds through the host-buffer entry point: p, v and gradients
     start in pinned host memory and p, v end there; every copy is inside the
@@ -536,6 +560,13 @@ def main():
             others[other.name] = {"gbs": ogbs, "frac_of_%s_peak" % peak_kind: ogbs / peak,
                                   "ms_per_step": osec / osteps * 1e3,
                                   "param_elements_per_s": other.n * osteps / osec, "steps": osteps}
+            if other.n <= 30_000_000 and not other.multi_tensor:
+                # Launch-bound size: also time the same rounds replayed from a CUDA
+                # graph (schedules encoded once at capture), i.e. without the host.
+                gms = time_graph_replay(odw, 100, 10)
+                others[other.name]["cuda_graph_replay"] = {
+                    "ms_per_step": gms, "gbs": obytes / osteps / (gms / 1e3) / 1e9,
+                    "note": "L2-resident working set: not an HBM figure"}
             del odw
             torch.cuda.empty_cache()
         out["other_workloads"] = others

@@ -236,3 +236,34 @@ def test_runs_on_a_side_stream_and_counts_launches(B):
         O.group_update_f32(p_np, v_np, g_np, [0, 1, 2], [1, 0], np.float32(0.1), 0.9, 1e-4)
     assert_matches(p, p_np, "p")
     assert_matches(v, v_np, "v")
+
+
+def test_rounds_captured_in_a_cuda_graph_replay_correctly(B):
+    """The flat entry point only enqueues one kernel on the given stream, so a
+    sequence of rounds can be captured once and replayed (launch-bound small
+    tensors).  Three rounds with different schedules, replayed twice."""
+    n = 65_537
+    (_, p), (_, v), grads = make_case(n, 4, torch.bfloat16, seed=41)
+    gl = [g for _, g in grads]
+    schedules = [([0, 2, 4], [0, 1, 2, 3]), ([0, 1, 2, 3, 4], [3, 1, 0, 2]), ([0, 4], [2, 3, 0, 1])]
+    p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+    g_np = [grad_to_numpy(g) for g in gl]
+    B.star_group_update(p, v, gl, *schedules[0], 0.1, 0.9, 1e-4)          # warm-up outside the capture
+    O.group_update_f32(p_np, v_np, g_np, *schedules[0], np.float32(0.1), 0.9, 1e-4)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for off, mem in schedules:
+                B.star_group_update(p, v, gl, off, mem, 0.1, 0.9, 1e-4)
+    # capturing does not execute: state is still the warm-up result
+    assert_matches(p, p_np, "p after capture")
+    for _ in range(2):
+        graph.replay()
+        for off, mem in schedules:
+            O.group_update_f32(p_np, v_np, g_np, off, mem, np.float32(0.1), 0.9, 1e-4)
+    torch.cuda.synchronize()
+    assert_matches(p, p_np, "p after replays")
+    assert_matches(v, v_np, "v after replays")
