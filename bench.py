@@ -449,7 +449,7 @@ def run_reference(args, rank: int):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": seconds / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": w.name, "model": w.model, "n": w.n, "W": w.W,
+        "data": "synthetic", "config": {"workload": w.name, "stands_for": w.model, "n": w.n, "W": w.W,
                                         "grad_dtype": w.grad_dtype, "sample_elements": n_sample},
         "param_elements_per_s": n_sample * args.steps / seconds,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
@@ -519,7 +519,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": seconds / args.steps * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "model": w.model, "n": w.n, "W": w.W, "grad_dtype": w.grad_dtype,
+        "config": {"workload": w.name, "stands_for": w.model, "n": w.n, "W": w.W, "grad_dtype": w.grad_dtype,
                    "tensors": len(w.sizes), "bytes_per_step": nbytes // args.steps,
                    "l2": "inputs larger than L2: %.0f MB per step, gradient buffer sets rotated: %d" % (
                        nbytes / args.steps / 1e6, len(dw.grad_sets)),
