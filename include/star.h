@@ -223,7 +223,7 @@ STAR_API star_status_t star_group_update(float *params, float *momentum, const v
 /* The same round with one learning rate per group, optional parameter
  * snapshots and a choice of the in-group summation order (sum_order; the tree
  * order keeps up to log2|G| partial sums per element in registers, runs at lower
- * occupancy and reaches about 60-75 % of the linear order's throughput).
+ * occupancy and reaches about 65-75 % of the linear order's throughput).
  *   lrs        : host, n_groups learning rates.  Section IV-C1 ("Scaling learning
  *                rate after switching") sets the rate of an update built from y
  *                gradient reports to (y / N) x the SSGD rate; the caller computes

@@ -114,6 +114,7 @@ constexpr int kVecBF16 = 8;
 constexpr int kVecF32 = 4;
 constexpr int kDepthVector = 4;
 constexpr int kDepthScalar = 4;
+constexpr int kDepthTree = 2;             // tree order with 4 or 6 levels: registers go to the pending partial sums
 constexpr int kVecBF16Half = 4;           // bf16 with buffers aligned for 16-byte state / 8-byte gradient accesses
 
 // Alignment of the buffers of a call: the smallest power of two (capped at 32)
@@ -243,7 +244,7 @@ template <typename G, int VEC, int TREE>
 star_status_t launch_flat_snapshot(const SnapshotArgs &args, cudaStream_t stream)
 {
     static Geometry cache[kMaxDevices];
-    constexpr int depth = VEC == 1 ? kDepthScalar : kDepthVector;
+    constexpr int depth = VEC == 1 ? kDepthScalar : (TREE > 2 ? kDepthTree : kDepthVector);
     auto kernel = star_update_flat_snapshot_kernel<G, VEC, depth, TREE>;
     int blocks = 0;
     cudaError_t e = resident_blocks(kernel, cache, &blocks);

@@ -209,7 +209,7 @@ struct NoSnapshot {
 // That is tree(first h) + tree(rest) with h the largest power of two below the
 // group size.  A group of c members needs ceil(log2(c)) pending levels of VEC
 // registers each, so the tree kernels are instantiated for 2, 4 and 6 levels
-// (groups of up to 4, 16 and 64 members) and compiled for 3, 2 and 2 resident
+// (groups of up to 4, 16 and 64 members) and compiled for 3, 3 and 2 resident
 // blocks; TREE is the number of levels, 0 = linear order.
 
 // Merge a new leaf with the pending partial sums of levels 0..LEVEL-1 and park
@@ -268,15 +268,23 @@ __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first,
                 } else if constexpr (TREE > 0) {
                     const int leaves_before = s.index_in_group[base + j];
                     if (gs == 0) {                   // not the last leaf: merge up to the first clear bit
-                        // A real (warp-uniform) branch per level: predicating all six
-                        // levels on every leaf made this path issue-bound.
-                        switch (__ffs(~leaves_before) - 1) {      // number of trailing set bits
-                        case 0: tree_merge<0, VEC>(pending, f); break;
-                        case 1: tree_merge<1, VEC>(pending, f); break;
-                        case 2: tree_merge<2, VEC>(pending, f); break;
-                        case 3: tree_merge<3, VEC>(pending, f); break;
-                        case 4: tree_merge<4, VEC>(pending, f); break;
-                        default: tree_merge<5, VEC>(pending, f); break;
+                        // A real (warp-uniform) branch per level, most frequent level
+                        // first: predicating all levels on every leaf made this path
+                        // issue-bound, and a jump table was slower than this chain.
+                        const int level = __ffs(~leaves_before) - 1;      // number of trailing set bits
+                        if (level == 0) {
+                            tree_merge<0, VEC>(pending, f);
+                        } else if (level == 1) {
+                            tree_merge<1, VEC>(pending, f);
+                        } else if constexpr (TREE > 2) {
+                            if (level == 2) {
+                                tree_merge<2, VEC>(pending, f);
+                            } else if (level == 3) {
+                                tree_merge<3, VEC>(pending, f);
+                            } else if constexpr (TREE > 4) {
+                                if (level == 4) tree_merge<4, VEC>(pending, f);
+                                else tree_merge<5, VEC>(pending, f);
+                            }
                         }
                     } else {                         // last leaf: fold every pending level
 #pragma unroll
@@ -364,7 +372,7 @@ struct StoreSnapshot {
 
 constexpr int tree_resident_blocks(int levels)
 {
-    return levels == 0 ? kResidentBlocks : levels <= 2 ? 3 : 2;
+    return levels == 0 ? kResidentBlocks : levels <= 4 ? 3 : 2;
 }
 
 template <typename G, int VEC, int DEPTH, int TREE>
