@@ -4,7 +4,7 @@
 // then walks the flattened schedule (all members of all groups, in order) in
 // chunks of DEPTH members: the DEPTH gradient loads of a chunk are issued back
 // to back before any of them is consumed, so each thread keeps
-// DEPTH * 16..32 bytes in flight on top of p and v.  Every group's update is
+// DEPTH * 8..16 bytes in flight on top of p and v.  Every group's update is
 // applied in registers; p and v are stored once.
 //
 // The arithmetic is the pinned binary32 sequence
@@ -56,7 +56,6 @@ template <> struct Raw<2>  { uint32_t w[1]; };
 template <> struct Raw<4>  { uint32_t w[1]; };
 template <> struct Raw<8>  { uint32_t w[2]; };
 template <> struct Raw<16> { uint32_t w[4]; };
-template <> struct Raw<32> { uint32_t w[8]; };
 
 template <int BYTES> __device__ __forceinline__ Raw<BYTES> load_stream(const void *p);
 
@@ -87,15 +86,6 @@ template <> __device__ __forceinline__ Raw<16> load_stream<16>(const void *p)
                  : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]) : "l"(p));
     return r;
 }
-template <> __device__ __forceinline__ Raw<32> load_stream<32>(const void *p)
-{
-    Raw<32> r;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]),
-                   "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7]) : "l"(p));
-    return r;
-}
-
 // p / v: VEC floats, through 4-, 16- or 32-byte accesses.
 template <int VEC> __device__ __forceinline__ void load_state(const float *src, float (&x)[VEC])
 {
