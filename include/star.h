@@ -228,11 +228,12 @@ STAR_API star_status_t star_group_update(float *params, float *momentum, const v
  *                rate after switching") sets the rate of an update built from y
  *                gradient reports to (y / N) x the SSGD rate; the caller computes
  *                the rates, the kernel applies lrs[k] in group k's update.
- *   snapshots  : NULL, or host array of n_groups device pointers (fp32, n
- *                elements each, entries may be NULL).  snapshots[k] receives the
- *                parameters as they stand right after group k's update -- the
+ *   snapshots  : NULL, or host array of n_groups device pointers (n elements of
+ *                snapshot_dtype each, entries may be NULL).  snapshots[k] receives
+ *                the parameters as they stand right after group k's update -- the
  *                copy the server sends back to that group's workers (Section II)
- *                -- written in the same pass (4 n more bytes of traffic each).
+ *                -- written in the same pass: fp32 (4 n more bytes of traffic
+ *                each) or rounded to bf16, nearest-even (2 n bytes each).
  *                Snapshot buffers must not overlap each other or any other
  *                buffer of the call.
  * Everything else as star_group_update.  One kernel launch. */
@@ -241,8 +242,8 @@ STAR_API star_status_t star_group_update_ex(float *params, float *momentum, cons
                                             const int32_t *group_offsets,
                                             const int32_t *group_members, int n_groups,
                                             const float *lrs, float mu, float wd,
-                                            float *const *snapshots, star_sum_order_t sum_order,
-                                            void *cuda_stream);
+                                            void *const *snapshots, star_dtype_t snapshot_dtype,
+                                            star_sum_order_t sum_order, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
  * Fused grouped update of a LIST of tensors (per-layer parameters) in one

@@ -72,6 +72,17 @@ static float widen_bf16(uint16_t h)
     return f;
 }
 
+/* binary32 -> bf16, round to nearest, ties to even; NaN stays NaN (quiet). */
+static uint16_t narrow_bf16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u)
+        return (uint16_t)((u >> 16) | 0x0040u);
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
 static float grad_at(const void *buf, int dtype, int64_t i)
 {
     if (dtype == ORACLE_DTYPE_BF16)
@@ -130,16 +141,18 @@ static int schedule_ok(const int32_t *group_offsets, const int32_t *group_member
  * of gradient reports y used by the update); pass the same value K times for
  * a single rate.  snapshots is NULL, or K pointers of which the non-NULL ones
  * receive the parameters as they stand right after that group's update: the
- * copy the PS sends back to the workers of that group (Section II).
+ * copy the PS sends back to the workers of that group (Section II), as
+ * binary32 (snapshot_dtype 0) or rounded to bf16 (snapshot_dtype 1).
  */
 int oracle_group_update_f32(float *params, float *momentum,
                             const void *const *grads, int W, int grad_dtype,
                             int64_t n, const int32_t *group_offsets,
                             const int32_t *group_members, int n_groups,
                             const float *lrs, float mu, float wd,
-                            float *const *snapshots, int sum_order)
+                            void *const *snapshots, int snapshot_dtype, int sum_order)
 {
-    if (!schedule_ok(group_offsets, group_members, n_groups, W) || sum_order < 0 || sum_order > 1)
+    if (!schedule_ok(group_offsets, group_members, n_groups, W) || sum_order < 0 || sum_order > 1 ||
+        snapshot_dtype < 0 || snapshot_dtype > 1)
         return 1;
     for (int64_t i = 0; i < n; ++i) {
         float p = params[i];
@@ -159,8 +172,12 @@ int oracle_group_update_f32(float *params, float *momentum,
             const float d = fmaf(wd, p, gbar);
             v = fmaf(mu, v, d);
             p = fmaf(-lrs[k], v, p);
-            if (snapshots && snapshots[k])
-                snapshots[k][i] = p;
+            if (snapshots && snapshots[k]) {
+                if (snapshot_dtype == ORACLE_DTYPE_BF16)
+                    ((uint16_t *)snapshots[k])[i] = narrow_bf16(p);
+                else
+                    ((float *)snapshots[k])[i] = p;
+            }
         }
         params[i] = p;
         momentum[i] = v;

@@ -51,7 +51,7 @@ def _load():
                   ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
                   ctypes.c_int, ctypes.c_void_p]
         lib.oracle_group_update_f32.argtypes = common + [
-            ctypes.c_float, ctypes.c_float, ctypes.c_void_p, ctypes.c_int]
+            ctypes.c_float, ctypes.c_float, ctypes.c_void_p, ctypes.c_int, ctypes.c_int]
         lib.oracle_group_update_f32.restype = ctypes.c_int
         lib.oracle_group_update_f64.argtypes = common + [
             ctypes.c_double, ctypes.c_double, ctypes.c_void_p, ctypes.c_int]
@@ -102,6 +102,7 @@ def _call(fn, real, params, momentum, grads, group_offsets, group_members, lrs, 
         if 0 <= w < W and grads[w] is None:
             raise ValueError("scheduled worker %d has no gradient buffer" % w)
     snap_ptrs = None
+    snap_kinds = set()
     if snapshots is not None:
         if len(snapshots) != K:
             raise ValueError("snapshots needs one entry (array or None) per group")
@@ -110,12 +111,21 @@ def _call(fn, real, params, momentum, grads, group_offsets, group_members, lrs, 
             if s is None:
                 snap_ptrs[k] = None
                 continue
-            if s.dtype != real or s.shape != (n,) or not s.flags.c_contiguous:
-                raise ValueError("snapshot %d has the wrong dtype or shape" % k)
+            if s.dtype == np.uint16 and real == np.float32:
+                snap_kinds.add(DTYPE_BF16)
+            elif s.dtype == real:
+                snap_kinds.add(DTYPE_F32)
+            else:
+                raise ValueError("snapshot %d has the wrong dtype" % k)
+            if s.shape != (n,) or not s.flags.c_contiguous:
+                raise ValueError("snapshot %d has the wrong shape" % k)
             snap_ptrs[k] = s.ctypes.data
+    if len(snap_kinds) > 1:
+        raise ValueError("snapshots must all have one dtype")
+    extra = [snap_kinds.pop() if snap_kinds else DTYPE_F32] if real == np.float32 else []
     rc = fn(params.ctypes.data, momentum.ctypes.data, ptrs, W, dt, n,
             off.ctypes.data, mem.ctypes.data, K, lr_arr.ctypes.data,
-            mu, wd, snap_ptrs, SUM_ORDERS[sum_order])
+            mu, wd, snap_ptrs, *extra, SUM_ORDERS[sum_order])
     if rc != 0:
         raise ValueError("schedule outside the definition (empty group, duplicate or "
                          "out-of-range member)")
@@ -127,7 +137,8 @@ def group_update_f32(params, momentum, grads, group_offsets, group_members, lrs,
 
     ``lrs`` is a scalar or one learning rate per group.  ``mu`` and ``wd`` are
     rounded to binary32 on the way in, as the C signature takes floats.
-    ``sum_order`` is "linear" (left to right) or "tree" (pairwise).
+    ``sum_order`` is "linear" (left to right) or "tree" (pairwise).  Snapshot
+    arrays are float32, or uint16 to receive the parameters rounded to bf16.
     """
     _call(_load().oracle_group_update_f32, np.float32, params, momentum, grads,
           group_offsets, group_members, lrs, float(np.float32(mu)), float(np.float32(wd)),

@@ -83,7 +83,7 @@ def _load() -> ctypes.CDLL:
                                        ctypes.c_size_t, c_vp, c_vp]
     lib.star_group_update_multi.argtypes = [c_vp, c_vp, c_vp, c_int, c_f, c_f, c_f, c_vp]
     lib.star_group_update_ex.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
-                                         c_vp, c_f, c_f, c_vp, c_int, c_vp]
+                                         c_vp, c_f, c_f, c_vp, c_int, c_int, c_vp]
     lib.star_group_update_ex.restype = c_int
     lib.star_cluster_iteration_times.argtypes = [c_vp, c_int, c_int, ctypes.c_double, c_vp, c_vp]
     lib.star_cluster_iteration_times.restype = c_int
@@ -313,9 +313,9 @@ def star_group_update_ex(params: torch.Tensor, momentum: torch.Tensor,
                          group_members: Sequence[int], lrs: Sequence[float], mu: float, wd: float,
                          snapshots: Optional[Sequence[Optional[torch.Tensor]]] = None,
                          sum_order: int = STAR_SUM_LINEAR, stream=None) -> None:
-    """The round with one learning rate per group; ``snapshots[k]`` (fp32 CUDA
-    tensor or None) receives the parameters right after group k's update;
-    ``sum_order`` is STAR_SUM_LINEAR or STAR_SUM_TREE."""
+    """The round with one learning rate per group; ``snapshots[k]`` (CUDA tensor,
+    all float32 or all bfloat16, or None) receives the parameters right after
+    group k's update; ``sum_order`` is STAR_SUM_LINEAR or STAR_SUM_TREE."""
     n = params.numel()
     p, v = _state(params, "params"), _state(momentum, "momentum")
     if momentum.numel() != n:
@@ -337,20 +337,25 @@ def star_group_update_ex(params: torch.Tensor, momentum: torch.Tensor,
     if len(lrs) != K:
         raise ValueError("need one learning rate per group")
     lr_arr = (ctypes.c_float * max(K, 1))(*lrs)
-    snap_arr = None
+    snap_arr, snap_dt = None, STAR_DTYPE_F32
     if snapshots is not None:
         if len(snapshots) != K:
             raise ValueError("snapshots needs one entry (tensor or None) per group")
         snap_arr = (ctypes.c_void_p * max(K, 1))()
+        kinds = set()
         for k, s in enumerate(snapshots):
             if s is None:
                 continue
-            if s.numel() != n:
-                raise ValueError("snapshot %d differs in size" % k)
-            snap_arr[k] = _state(s, "snapshot")
+            if s.numel() != n or not s.is_cuda or not s.is_contiguous():
+                raise ValueError("snapshot %d must be a contiguous CUDA tensor of %d elements" % (k, n))
+            kinds.add(_grad_dtype(s))
+            snap_arr[k] = s.data_ptr()
+        if len(kinds) > 1:
+            raise TypeError("snapshots differ in dtype")
+        snap_dt = kinds.pop() if kinds else STAR_DTYPE_F32
     _check(_lib.star_group_update_ex(p, v, ptrs, W, STAR_DTYPE_F32 if dt is None else dt, n,
                                      _i32(group_offsets), _i32(group_members), K, lr_arr, mu, wd,
-                                     snap_arr, sum_order, _stream(stream)), "star_group_update_ex")
+                                     snap_arr, snap_dt, sum_order, _stream(stream)), "star_group_update_ex")
 
 
 def star_multi_workspace_bytes(sizes: Sequence[int], W: int) -> int:

@@ -286,10 +286,11 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
                                               int W, star_dtype_t grad_dtype, int64_t n,
                                               const int32_t *group_offsets, const int32_t *group_members,
                                               int n_groups, const float *lrs, float mu, float wd,
-                                              float *const *snapshots, star_sum_order_t sum_order,
-                                              void *cuda_stream)
+                                              void *const *snapshots, star_dtype_t snapshot_dtype,
+                                              star_sum_order_t sum_order, void *cuda_stream)
 {
     if (sum_order != STAR_SUM_LINEAR && sum_order != STAR_SUM_TREE) return STAR_ERR_INVALID_ARG;
+    if (snapshot_dtype != STAR_DTYPE_F32 && snapshot_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
     if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
     SnapshotArgs sargs;
     FlatArgs &args = sargs.flat;
@@ -302,18 +303,23 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
     const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
     const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
     std::memset(sargs.snapshots, 0, sizeof sargs.snapshots);
+    sargs.snapshot_bf16 = snapshot_dtype == STAR_DTYPE_BF16 ? 1 : 0;
+    const size_t snap_elem = snapshot_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const size_t snap_bytes = static_cast<size_t>(n) * snap_elem;
     bool any_snapshot = false;
     for (int k = 0; snapshots && k < n_groups; ++k) {
-        float *snap = snapshots[k];
+        void *snap = snapshots[k];
         if (!snap) continue;
-        if (!aligned(snap, 4)) return STAR_ERR_INVALID_ARG;
-        if (overlaps(snap, state_bytes, params, state_bytes) || overlaps(snap, state_bytes, momentum, state_bytes))
+        if (!aligned(snap, snap_elem)) return STAR_ERR_INVALID_ARG;
+        if (overlaps(snap, snap_bytes, params, state_bytes) || overlaps(snap, snap_bytes, momentum, state_bytes))
             return STAR_ERR_INVALID_ARG;
         for (int j = 0; j < args.sched.n_slots; ++j)
-            if (overlaps(snap, state_bytes, args.grads[args.sched.member[j]], grad_bytes)) return STAR_ERR_INVALID_ARG;
+            if (overlaps(snap, snap_bytes, args.grads[args.sched.member[j]], grad_bytes)) return STAR_ERR_INVALID_ARG;
         for (int l = 0; l < k; ++l)
-            if (snapshots[l] && overlaps(snap, state_bytes, snapshots[l], state_bytes)) return STAR_ERR_INVALID_ARG;
-        align.add_state(snap);
+            if (snapshots[l] && overlaps(snap, snap_bytes, snapshots[l], snap_bytes)) return STAR_ERR_INVALID_ARG;
+        // a bf16 snapshot moves half the bytes: 16-byte alignment serves the full vector width
+        if (snapshot_dtype == STAR_DTYPE_BF16) align.state = std::min(align.state, 2 * Alignment::of(snap));
+        else align.add_state(snap);
         sargs.snapshots[group_offsets[k + 1] - 1] = snap;
         any_snapshot = true;
     }

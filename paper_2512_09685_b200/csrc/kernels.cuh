@@ -348,15 +348,47 @@ star_update_flat_kernel(const __grid_constant__ FlatArgs a)
 // workers) and the tree summation order.
 struct SnapshotArgs {
     FlatArgs flat;
-    float *snapshots[kMaxWorkers];     // indexed by closing slot
+    void *snapshots[kMaxWorkers];      // indexed by closing slot; fp32 or bf16 buffers
+    int32_t snapshot_bf16;             // 0: snapshots are fp32, 1: rounded to bf16
 };
+
+// binary32 -> bf16 bit pattern: round to nearest, ties to even; NaN stays a
+// (quiet) NaN.
+__device__ __forceinline__ uint32_t narrow_bf16(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (u >> 16) | 0x0040u;
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return u >> 16;
+}
+
+// VEC parameters as bf16: one 2-, 8- or 16-byte store.
+template <int VEC> __device__ __forceinline__ void store_bf16(uint16_t *dst, const float (&x)[VEC])
+{
+    if constexpr (VEC == 1) {
+        *dst = static_cast<uint16_t>(narrow_bf16(x[0]));
+    } else {
+        uint32_t w[VEC / 2];
+#pragma unroll
+        for (int e = 0; e < VEC / 2; ++e) w[e] = narrow_bf16(x[2 * e]) | (narrow_bf16(x[2 * e + 1]) << 16);
+        if constexpr (VEC == 8) {
+            asm volatile("st.global.L1::no_allocate.v4.u32 [%4], {%0,%1,%2,%3};"
+                         :: "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "l"(dst) : "memory");
+        } else {
+            static_assert(VEC == 4, "bf16 snapshot stores exist for 1, 4 and 8 elements");
+            asm volatile("st.global.L1::no_allocate.v2.u32 [%2], {%0,%1};" :: "r"(w[0]), "r"(w[1]), "l"(dst) : "memory");
+        }
+    }
+}
 
 struct StoreSnapshot {
     const SnapshotArgs *a;
     template <int VEC> __device__ __forceinline__ void operator()(int slot, int64_t first, const float (&p)[VEC]) const
     {
-        float *dst = a->snapshots[slot];
-        if (dst != nullptr) store_state<VEC>(dst + first, p);
+        void *dst = a->snapshots[slot];
+        if (dst == nullptr) return;
+        if (a->snapshot_bf16) store_bf16<VEC>(static_cast<uint16_t *>(dst) + first, p);
+        else store_state<VEC>(static_cast<float *>(dst) + first, p);
     }
 };
 

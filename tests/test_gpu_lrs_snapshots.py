@@ -146,3 +146,44 @@ def test_tree_and_linear_orders_differ_only_in_rounding(B):
     assert float((p - q).abs().max()) <= 8 * 2.0 ** -24 * 0.1
     with pytest.raises(B.StarError):
         B.star_group_update_ex(p, v, grads, off, mem, [0.1], 0.9, 1e-4, sum_order=5)
+
+
+@pytest.mark.parametrize("n", [3, 4099, 500_001])
+def test_bf16_snapshots_match_oracle(B, n):
+    W = 6
+    p, v, grads = case(n, W, torch.bfloat16, seed=n + 1)
+    # plant exact ties for the narrowing in the first snapshot: p' = p - lr * v' with v' = g, lr = 1
+    off, mem = [0, 2, 6], [1, 0, 5, 4, 3, 2]
+    p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+    g_np = [grad_to_numpy(g) for g in grads]
+    want = [np.zeros(n, np.uint16), np.zeros(n, np.uint16)]
+    O.group_update_f32(p_np, v_np, g_np, off, mem, np.array([0.1, 0.05], np.float32), 0.9, 1e-3, snapshots=want)
+    snaps = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    B.star_group_update_ex(p, v, grads, off, mem, [0.1, 0.05], 0.9, 1e-3, snapshots=snaps)
+    torch.cuda.synchronize()
+    assert_matches(p, p_np, "params")
+    for k in range(2):
+        got = snaps[k].cpu().view(torch.int16).numpy().view(np.uint16)
+        assert np.array_equal(got, want[k]), "snapshot %d" % k
+    assert torch.equal(snaps[1], p.to(torch.bfloat16))            # torch's cast rounds the same way
+
+
+def test_bf16_snapshot_narrowing_on_ties_and_extremes(B):
+    """Zero gradients and momentum hold the parameters still: the snapshot is the
+    narrowing of the input, compared with the oracle and with torch's cast."""
+    from tests.test_oracle_pins import bf16_snapshot_probe_values
+    x = bf16_snapshot_probe_values()
+    n = x.size
+    p = torch.from_numpy(x.copy()).cuda()
+    v = torch.zeros(n, device="cuda")
+    g = torch.zeros(n, device="cuda")
+    for misalign in (0, 1):
+        raw = torch.zeros(n + 1, dtype=torch.bfloat16, device="cuda")
+        snap = raw[misalign: misalign + n]
+        B.star_group_update_ex(p, v, [g], [0, 1], [0], [0.1], 0.9, 0.0, snapshots=[snap])
+        torch.cuda.synchronize()
+        assert torch.equal(snap.view(torch.int16), torch.from_numpy(x).cuda().to(torch.bfloat16).view(torch.int16))
+    want = np.zeros(n, np.uint16)
+    O.group_update_f32(x.copy(), np.zeros(n, np.float32), [np.zeros(n, np.float32)], [0, 1], [0], 0.1, 0.9, 0.0,
+                       snapshots=[want])
+    assert np.array_equal(snap.cpu().view(torch.int16).numpy().view(np.uint16), want)

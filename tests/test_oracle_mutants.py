@@ -13,7 +13,8 @@ import torch
 
 from oracle import star_oracle as O
 from tests import exact_arith as X
-from tests.test_oracle_pins import _read_golden, all_schedules, bf16_bits, bf16_values, csr
+from tests.test_oracle_pins import (_read_golden, all_schedules, bf16_bits, bf16_snapshot_probe_values,
+                                    bf16_values, csr)
 
 SRC = os.path.join(os.path.dirname(O.__file__), "star_oracle.c")
 
@@ -39,8 +40,9 @@ MUTANTS = {
     "tree_drops_the_right_half": ("tree_sum_f32(grads, dtype, members + h, count - h, i);",
                                   "tree_sum_f32(grads, dtype, members + h, 1, i);"),
     "bf16_widened_wrongly": ("uint32_t u = (uint32_t)h << 16;", "uint32_t u = (uint32_t)h << 15;"),
-    "snapshot_of_the_final_state_only": ("snapshots[k][i] = p;\n        }\n        params[i] = p;",
-                                         "snapshots[k][i] = params[i];\n        }\n        params[i] = p;"),
+    "snapshot_of_the_old_state": ("((float *)snapshots[k])[i] = p;", "((float *)snapshots[k])[i] = params[i];"),
+    "bf16_snapshot_truncated_not_rounded": ("u += 0x7fffu + ((u >> 16) & 1u);", "u += 0u;"),
+    "bf16_snapshot_ties_away": ("u += 0x7fffu + ((u >> 16) & 1u);", "u += 0x8000u;"),
     "dampened_momentum": ("v = fmaf(mu, v, d);", "v = fmaf(mu, v, (1.0f - mu) * d);"),
 }
 
@@ -57,7 +59,8 @@ def build_mutant(tmp_path, name):
     lib = ctypes.CDLL(lib_path)
     common = [ctypes.c_void_p] * 3 + [ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_void_p,
                                       ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
-    lib.oracle_group_update_f32.argtypes = common + [ctypes.c_float, ctypes.c_float, ctypes.c_void_p, ctypes.c_int]
+    lib.oracle_group_update_f32.argtypes = common + [ctypes.c_float, ctypes.c_float, ctypes.c_void_p, ctypes.c_int,
+                                                     ctypes.c_int]
     lib.oracle_group_update_f32.restype = ctypes.c_int
 
     def update(p, v, grads, off, mem, lrs, mu, wd, snapshots=None, sum_order="linear"):
@@ -119,6 +122,13 @@ def pins_accept(update) -> bool:
                 X.to_fraction(np.float32(1e-3)), tree=True)
             if X.to_fraction(p[i]) != pe or X.to_fraction(v[i]) != ve:
                 return False
+    # bf16 snapshots against PyTorch's cast (parameters held still by zero gradients)
+    x = bf16_snapshot_probe_values()
+    snap = np.zeros(x.size, np.uint16)
+    update(x.copy(), np.zeros(x.size, np.float32), [np.zeros(x.size, np.float32)], [0, 1], [0], 0.1, 0.9, 0.0,
+           snapshots=[snap])
+    if not np.array_equal(snap, torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)):
+        return False
     # PyTorch's SGD, two rounds of three groups (fp32 state: agreement to rounding)
     n = 64
     p0 = rng.normal(0, 0.05, n).astype(np.float32)

@@ -146,6 +146,42 @@ def test_tree_and_linear_orders_agree_up_to_rounding_and_exactly_for_small_group
         assert np.max(np.abs(x - P)) <= 16 * 2.0 ** -24 * 0.2
 
 
+def bf16_snapshot_probe_values():
+    """fp32 values that exercise the narrowing: random, exact ties with even and
+    odd upper halves, just above / below ties, overflow to infinity, subnormals,
+    signed zeros (infinite parameters turn into NaN through wd * p and cannot be
+    held still)."""
+    rng = np.random.default_rng(17)
+    vals = [rng.normal(0, 1, 4096).astype(np.float32),
+            (rng.normal(0, 1, 512) * 10.0 ** rng.integers(-30, 30, 512)).astype(np.float32)]
+    upper = rng.integers(0x0001, 0x7F7F, 2048).astype(np.uint32) << 16
+    for low in (0x8000, 0x7FFF, 0x8001, 0x0001, 0xFFFF):
+        vals.append((upper | low).view(np.float32))
+        vals.append((upper | low | 0x80000000).view(np.float32))
+    special = np.array([0x7F7FFFFF, 0x7F7F8000, 0x7F7F7FFF, 0x00000001, 0x00008000, 0x00018000, 0x00007FFF,
+                        0x00000000, 0x80000000], np.uint32).view(np.float32)
+    vals.append(special)
+    return np.concatenate(vals)
+
+
+def test_bf16_snapshots_round_to_nearest_even_like_torch():
+    """With zero gradients and zero momentum the parameters do not move, so the
+    bf16 snapshot is the narrowing of the input: compare with PyTorch's cast."""
+    x = bf16_snapshot_probe_values()
+    n = x.size
+    p, v = x.copy(), np.zeros(n, np.float32)
+    snap = np.zeros(n, np.uint16)
+    O.group_update_f32(p, v, [np.zeros(n, np.float32)], [0, 1], [0], 0.1, 0.9, 0.0, snapshots=[snap])
+    assert np.array_equal(p.view(np.uint32), x.view(np.uint32))
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(snap, want)
+    nan = np.array([np.nan], np.float32)
+    s1 = np.zeros(1, np.uint16)
+    O.group_update_f32(nan.copy(), np.zeros(1, np.float32), [np.zeros(1, np.float32)], [0, 1], [0], 0.1, 0.9, 0.0,
+                       snapshots=[s1])
+    assert np.isnan(bf16_values(s1))[0]
+
+
 # --------------------------------------------------------------------------
 # 2. exact-rational brute force: every schedule over W<=4, tiny n
 # --------------------------------------------------------------------------
