@@ -296,6 +296,14 @@ STAR_API star_status_t star_group_update_multi(const star_multi_plan_t *plan,
                                       int n_groups, float lr, float mu, float wd,
                                       void *cuda_stream);
 
+/* The tensor-list round with one learning rate per group (lrs: host, n_groups
+ * values; Section IV-C1 rate scaling).  Otherwise as star_group_update_multi. */
+STAR_API star_status_t star_group_update_multi_lrs(const star_multi_plan_t *plan,
+                                                   const int32_t *group_offsets,
+                                                   const int32_t *group_members, int n_groups,
+                                                   const float *lrs, float mu, float wd,
+                                                   void *cuda_stream);
+
 /* ---------------------------------------------------------------------------
  * Fused grouped update with the state and the gradients in HOST memory (the
  * paper's parameter server keeps its parameter and gradient copies in host

@@ -82,6 +82,8 @@ def _load() -> ctypes.CDLL:
     lib.star_multi_prepare.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp,
                                        ctypes.c_size_t, c_vp, c_vp]
     lib.star_group_update_multi.argtypes = [c_vp, c_vp, c_vp, c_int, c_f, c_f, c_f, c_vp]
+    lib.star_group_update_multi_lrs.argtypes = [c_vp, c_vp, c_vp, c_int, c_vp, c_f, c_f, c_vp]
+    lib.star_group_update_multi_lrs.restype = c_int
     lib.star_group_update_ex.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
                                          c_vp, c_f, c_f, c_vp, c_int, c_int, c_vp]
     lib.star_group_update_ex.restype = c_int
@@ -411,6 +413,17 @@ def star_group_update_multi(plan: star_multi_plan_t, group_offsets: Sequence[int
     K = len(group_offsets) - 1 if len(group_offsets) else 0
     _check(_lib.star_group_update_multi(ctypes.byref(plan), _i32(group_offsets), _i32(group_members),
                                         K, lr, mu, wd, _stream(stream)), "star_group_update_multi")
+
+
+def star_group_update_multi_lrs(plan: star_multi_plan_t, group_offsets: Sequence[int],
+                                group_members: Sequence[int], lrs: Sequence[float], mu: float, wd: float,
+                                stream=None) -> None:
+    K = len(group_offsets) - 1 if len(group_offsets) else 0
+    if len(lrs) != K:
+        raise ValueError("need one learning rate per group")
+    _check(_lib.star_group_update_multi_lrs(ctypes.byref(plan), _i32(group_offsets), _i32(group_members), K,
+                                            (ctypes.c_float * max(K, 1))(*lrs), mu, wd, _stream(stream)),
+           "star_group_update_multi_lrs")
 
 
 def star_host_workspace_bytes(max_scheduled: int, grad_dtype: torch.dtype, chunk_elements: int) -> int:

@@ -503,15 +503,41 @@ extern "C" star_status_t star_multi_prepare(int n_tensors, float *const *params,
     return STAR_OK;
 }
 
+namespace {
+
+star_status_t update_multi(const star_multi_plan_t *plan, const int32_t *group_offsets,
+                           const int32_t *group_members, int n_groups, float lr, const float *lrs, float mu,
+                           float wd, void *cuda_stream);
+
+}  // namespace
+
 extern "C" star_status_t star_group_update_multi(const star_multi_plan_t *plan,
                                                  const int32_t *group_offsets, const int32_t *group_members,
                                                  int n_groups, float lr, float mu, float wd,
                                                  void *cuda_stream)
 {
+    return update_multi(plan, group_offsets, group_members, n_groups, lr, nullptr, mu, wd, cuda_stream);
+}
+
+extern "C" star_status_t star_group_update_multi_lrs(const star_multi_plan_t *plan,
+                                                     const int32_t *group_offsets,
+                                                     const int32_t *group_members, int n_groups,
+                                                     const float *lrs, float mu, float wd, void *cuda_stream)
+{
+    if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
+    return update_multi(plan, group_offsets, group_members, n_groups, 0.0f, lrs, mu, wd, cuda_stream);
+}
+
+namespace {
+
+star_status_t update_multi(const star_multi_plan_t *plan, const int32_t *group_offsets,
+                           const int32_t *group_members, int n_groups, float lr, const float *lrs, float mu,
+                           float wd, void *cuda_stream)
+{
     if (!plan) return STAR_ERR_NULL_POINTER;
     if (plan->magic != kPlanMagic || !plan->d_workspace) return STAR_ERR_INVALID_ARG;
     MultiArgs args;
-    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, plan->W, lr, &args.sched, nullptr);
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, plan->W, lr, &args.sched, lrs);
     if (st != STAR_OK) return st;
     if (plan->n_tiles == 0 || n_groups == 0) return STAR_OK;
     for (int j = 0; j < args.sched.n_slots; ++j)
@@ -532,6 +558,8 @@ extern "C" star_status_t star_group_update_multi(const star_multi_plan_t *plan,
     if (dt == STAR_DTYPE_F32) return launch_multi<GradF32, kVecF32>(args, stream);
     return STAR_ERR_INVALID_ARG;
 }
+
+}  // namespace
 
 // ---------------------------------------------------------------------------
 // Host-resident state and gradients: chunked, double-buffered streaming.

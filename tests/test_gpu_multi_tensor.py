@@ -107,3 +107,21 @@ def test_list_errors(B):
     assert not torch.equal(torch.cat(params), p0)
     empty_plan = B.star_multi_prepare([], [], [[] for _ in range(W)], ws)
     B.star_group_update_multi(empty_plan, [0, 1], [0], 0.1, 0.9, 0.0)
+
+
+def test_list_round_with_per_group_rates(B):
+    W, sizes = 4, [5000, 3, 70_001, 2048]
+    params, momentum, grads = build(sizes, W, torch.bfloat16, seed=8)
+    ws = torch.empty(B.star_multi_workspace_bytes(sizes, W), dtype=torch.uint8, device="cuda")
+    plan = B.star_multi_prepare(params, momentum, grads, ws)
+    off, mem, lrs = [0, 1, 4], [2, 0, 1, 3], [0.025, 0.075]
+    p_np = torch.cat(params).cpu().numpy().copy()
+    v_np = torch.cat(momentum).cpu().numpy().copy()
+    g_np = [grad_to_numpy(torch.cat(grads[w])) for w in range(W)]
+    O.group_update_f32(p_np, v_np, g_np, off, mem, np.array(lrs, np.float32), 0.9, 0.01)
+    B.star_group_update_multi_lrs(plan, off, mem, lrs, 0.9, 0.01)
+    torch.cuda.synchronize()
+    assert_matches(torch.cat(params), p_np, "params")
+    assert_matches(torch.cat(momentum), v_np, "momentum")
+    with pytest.raises(ValueError):
+        B.star_group_update_multi_lrs(plan, off, mem, [0.1], 0.9, 0.01)
