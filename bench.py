@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # workload, with the SHA-256 of the kernel sources the capture was taken on:
 # once the sources differ the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "cfg1_resnet50": (787.8e6, "fe20bb1d94b859b7b39617a463a17061429140ad8ddc23edc733d7b3f914fa8e"),
+    "cfg1_resnet50": (787.5e6, "5af0f5bea2e04724fc0e59d8d62e7846f850f970888230a50ffaad3a332b7fd5"),
 }
 
 
