@@ -267,3 +267,45 @@ def test_rounds_captured_in_a_cuda_graph_replay_correctly(B):
     torch.cuda.synchronize()
     assert_matches(p, p_np, "p after replays")
     assert_matches(v, v_np, "v after replays")
+
+
+def test_concurrent_host_threads_on_their_own_streams(B):
+    """The library keeps per-device launch geometry in shared caches; two host
+    threads issuing rounds on their own streams and tensors must not disturb
+    each other."""
+    import threading
+    n, rounds = 40_003, 25
+    cases = []
+    for t in range(2):
+        (_, p), (_, v), grads = make_case(n, 3, torch.bfloat16 if t == 0 else torch.float32, seed=50 + t)
+        cases.append((p, v, [g for _, g in grads], ([0, 1, 3], [2, 0, 1]) if t == 0 else ([0, 3], [1, 2, 0])))
+    expected = []
+    for p, v, gl, (off, mem) in cases:
+        p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+        g_np = [grad_to_numpy(g) for g in gl]
+        for _ in range(rounds):
+            O.group_update_f32(p_np, v_np, g_np, off, mem, np.float32(0.05), 0.9, 1e-4)
+        expected.append((p_np, v_np))
+    torch.cuda.synchronize()
+    errors = []
+
+    def worker(idx):
+        try:
+            p, v, gl, (off, mem) = cases[idx]
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                for _ in range(rounds):
+                    B.star_group_update(p, v, gl, off, mem, 0.05, 0.9, 1e-4)
+            stream.synchronize()
+        except Exception as exc:                       # surfaced below
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for (p, v, _, _), (p_np, v_np) in zip(cases, expected):
+        assert_matches(p, p_np, "params")
+        assert_matches(v, v_np, "momentum")
