@@ -309,3 +309,29 @@ def test_concurrent_host_threads_on_their_own_streams(B):
     for (p, v, _, _), (p_np, v_np) in zip(cases, expected):
         assert_matches(p, p_np, "params")
         assert_matches(v, v_np, "momentum")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_sparse_gradients_with_exact_and_signed_zeros(B, dtype):
+    """Group sums that are exactly +0 or -0 (unused rows, dead units) take a
+    shortcut around the division in the kernel: the mean must still be the
+    IEEE quotient, sign of zero included."""
+    n, W = 50_001, 6
+    (_, p), (_, v), grads = make_case(n, W, dtype, seed=61)
+    gl = [g for _, g in grads]
+    g = torch.Generator(device="cuda").manual_seed(62)
+    keep = torch.rand(n, generator=g, device="cuda") < 0.3          # 70 % of the elements: all workers zero
+    negz = torch.rand(n, generator=g, device="cuda") < 0.5
+    for x in gl:
+        x.mul_(keep.to(x.dtype))
+        x.copy_(torch.where(~keep & negz, torch.full_like(x, -0.0), x))
+    gl[2][::7] = 0.0                                                 # mixed signs of zero inside a group
+    p[::11] = 0.0
+    off, mem = [0, 3, 4, 6], [0, 1, 2, 3, 4, 5]
+    for wd in (0.0, 1e-4):
+        q, u = p.clone(), v.clone().zero_()
+        want_p, want_v = run_both(B, q, u, gl, off, mem, 0.1, 0.0 if wd == 0.0 else 0.9, wd)
+        assert_matches(q, want_p, "p wd=%g" % wd)
+        assert_matches(u, want_v, "v wd=%g" % wd)
+        assert np.array_equal(np.signbit(u.cpu().numpy()), np.signbit(want_v))
+        assert np.array_equal(np.signbit(q.cpu().numpy()), np.signbit(want_p))
