@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # workload, with the SHA-256 of the kernel sources the capture was taken on:
 # once the sources differ the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "cfg1_resnet50": (787.5e6, "5af0f5bea2e04724fc0e59d8d62e7846f850f970888230a50ffaad3a332b7fd5"),
+    "cfg1_resnet50": (790.9e6, "f5e911d974634f5eb3fd6156f6e14ba3e7e39ba3c74004c57323496e84f0320a"),
 }
 
 

@@ -114,6 +114,7 @@ constexpr int kVecBF16 = 8;
 constexpr int kVecF32 = 4;
 constexpr int kDepthVector = 4;
 constexpr int kDepthScalar = 4;
+constexpr int kDepthNarrow = 8;           // flat kernels whose gradient loads are narrower than 16 bytes
 constexpr int kDepthTree = 2;             // tree order with 4 or 6 levels: registers go to the pending partial sums
 constexpr int kVecBF16Half = 4;           // bf16 with buffers aligned for 16-byte state / 8-byte gradient accesses
 
@@ -149,7 +150,8 @@ template <typename G, int VEC>
 star_status_t launch_flat(const FlatArgs &args, cudaStream_t stream)
 {
     static Geometry cache[kMaxDevices];
-    constexpr int depth = VEC == 1 ? kDepthScalar : kDepthVector;
+    // Narrow loads (element by element, half-width bf16) keep more of them in flight.
+    constexpr int depth = VEC * G::kBytes >= 16 ? kDepthVector : kDepthNarrow;
     auto kernel = star_update_flat_kernel<G, VEC, depth>;
     int blocks = 0;
     cudaError_t e = resident_blocks(kernel, cache, &blocks);
