@@ -60,10 +60,17 @@ class star_multi_plan_t(ctypes.Structure):
 
 
 def _load() -> ctypes.CDLL:
-    if not os.path.exists(LIB_PATH):
-        raise ImportError(
-            "%s is missing: build it with `python -m paper_2512_09685_b200.build` "
-            "(there is no CPU fallback)" % LIB_PATH)
+    # (Re)build in-tree when the library is missing or older than its sources and
+    # nvcc is at hand; otherwise fail loudly: there is no CPU fallback.
+    try:
+        from . import build as _build
+        if _build.is_stale():
+            _build.build()
+    except Exception as exc:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                "%s is missing and could not be built (%s): run "
+                "`python -m paper_2512_09685_b200.build`; there is no CPU fallback" % (LIB_PATH, exc))
     lib = ctypes.CDLL(LIB_PATH)
     c_int, c_i64, c_vp, c_f = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float
     lib.star_status_string.argtypes = [c_int]
