@@ -55,6 +55,26 @@
  * library SGD optimizer of PyTorch in fp64, SSGD == one mean update, fused K
  * groups == K single-group calls, member-permutation invariance.
  *
+ * All-reduce architecture (Section IV-B, paragraph "All-reduce architecture";
+ * Section IV-C1, Eq. 3).  x stragglers leave the ring and report to a parent
+ * each; a parent adds the gradients of its children (those that reported
+ * before it stopped waiting) to its own and hands the aggregate to the ring;
+ * the ring sums the aggregates of its members; the update uses the gradients
+ * of N - x + q workers.  Two functions state the arithmetic of that round:
+ *   oracle_group_reduce_f32        what a parent forwards: the binary32 sum of
+ *                                  the listed buffers (own gradient first,
+ *                                  then the children), left to right or
+ *                                  pairwise, stored as binary32 or rounded to
+ *                                  bf16.
+ *   oracle_update_from_sums_f32    one update from R partial sums: they are
+ *                                  added left to right in the listed (ring)
+ *                                  order, the mean divides by the number of
+ *                                  gradient reports behind them (N - x + q,
+ *                                  the batch Eq. 3 counts), then the three
+ *                                  fused multiply-adds of a group update.
+ * The paper fixes neither order; oracle/all_reduce.py composes the two into a
+ * round and states the reading.  Pins: tests/test_all_reduce_oracle.py.
+ *
  * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC
  */
 #include <math.h>
@@ -218,6 +238,77 @@ int oracle_group_update_f64(double *params, double *momentum,
         }
         params[i] = p;
         momentum[i] = v;
+    }
+    return 0;
+}
+
+/* 1 if members[0..count) are distinct workers in [0, W), count >= 1. */
+static int members_ok(const int32_t *members, int count, int W)
+{
+    if (count < 1 || !members)
+        return 0;
+    for (int j = 0; j < count; ++j) {
+        if (members[j] < 0 || members[j] >= W)
+            return 0;
+        for (int l = 0; l < j; ++l)
+            if (members[l] == members[j])
+                return 0;
+    }
+    return 1;
+}
+
+/*
+ * Section IV-B, all-reduce architecture: a parent aggregates "the gradients
+ * from its children and its own gradients".  out[i] = g[m_0][i] + g[m_1][i] +
+ * ... in binary32, in the listed order (sum_order 0) or pairwise (sum_order
+ * 1, as tree_sum_f32 above); out is binary32 (out_dtype 0) or the sum rounded
+ * to bf16, nearest even (out_dtype 1).  Returns 0, or 1 for arguments outside
+ * the definition.
+ */
+int oracle_group_reduce_f32(void *out, int out_dtype, const void *const *grads, int W, int grad_dtype,
+                            int64_t n, const int32_t *members, int count, int sum_order)
+{
+    if (!members_ok(members, count, W) || sum_order < 0 || sum_order > 1 || out_dtype < 0 || out_dtype > 1)
+        return 1;
+    for (int64_t i = 0; i < n; ++i) {
+        float s;
+        if (sum_order == 1) {
+            s = tree_sum_f32(grads, grad_dtype, members, count, i);
+        } else {
+            s = grad_at(grads[members[0]], grad_dtype, i);
+            for (int j = 1; j < count; ++j)
+                s = s + grad_at(grads[members[j]], grad_dtype, i);
+        }
+        if (out_dtype == ORACLE_DTYPE_BF16)
+            ((uint16_t *)out)[i] = narrow_bf16(s);
+        else
+            ((float *)out)[i] = s;
+    }
+    return 0;
+}
+
+/*
+ * Section IV-B / Eq. 3: the one update of an all-reduce round.  sums[0..R) are
+ * the binary32 aggregates of the R ring members in ring order; n_reports is
+ * the number of gradient reports they contain together (N - x + q >= R).
+ *     s    = sums[0][i] + sums[1][i] + ...     left to right
+ *     gbar = s / n_reports
+ *     d = fma(wd, p, gbar) ; v = fma(mu, v, d) ; p = fma(-lr, v, p)
+ */
+int oracle_update_from_sums_f32(float *params, float *momentum, const float *const *sums, int R, int64_t n,
+                                int n_reports, float lr, float mu, float wd)
+{
+    if (R < 1 || n_reports < R || !sums)
+        return 1;
+    for (int64_t i = 0; i < n; ++i) {
+        float s = sums[0][i];
+        for (int r = 1; r < R; ++r)
+            s = s + sums[r][i];
+        const float gbar = s / (float)n_reports;
+        const float d = fmaf(wd, params[i], gbar);
+        const float v = fmaf(mu, momentum[i], d);
+        momentum[i] = v;
+        params[i] = fmaf(-lr, v, params[i]);
     }
     return 0;
 }

@@ -56,6 +56,14 @@ def _load():
         lib.oracle_group_update_f64.argtypes = common + [
             ctypes.c_double, ctypes.c_double, ctypes.c_void_p, ctypes.c_int]
         lib.oracle_group_update_f64.restype = ctypes.c_int
+        lib.oracle_group_reduce_f32.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_int,
+                                                ctypes.c_int, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int,
+                                                ctypes.c_int]
+        lib.oracle_group_reduce_f32.restype = ctypes.c_int
+        lib.oracle_update_from_sums_f32.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                                    ctypes.c_int, ctypes.c_int64, ctypes.c_int,
+                                                    ctypes.c_float, ctypes.c_float, ctypes.c_float]
+        lib.oracle_update_from_sums_f32.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -150,3 +158,50 @@ def group_update_f64(params, momentum, grads, group_offsets, group_members, lrs,
     """Binary64 shadow of the same loop, in place on float64 arrays."""
     _call(_load().oracle_group_update_f64, np.float64, params, momentum, grads,
           group_offsets, group_members, lrs, float(mu), float(wd), snapshots, sum_order)
+
+
+def group_reduce_f32(grads, members, out_dtype="f32", sum_order="linear") -> np.ndarray:
+    """Binary32 sum of ``grads[m]`` for m in ``members`` (listed order or
+    pairwise): what a parent of the all-reduce architecture forwards.  Returns
+    a float32 array, or uint16 bf16 bit patterns for ``out_dtype="bf16"``."""
+    W = len(grads)
+    dt = _grad_dtype(grads)
+    n = next(g for g in grads if g is not None).shape[0]
+    ptrs = (ctypes.c_void_p * max(W, 1))()
+    for w, g in enumerate(grads):
+        if g is None:
+            continue
+        if g.shape != (n,) or not g.flags.c_contiguous:
+            raise ValueError("gradient %d must be contiguous with %d elements" % (w, n))
+        ptrs[w] = g.ctypes.data
+    mem = np.ascontiguousarray(members, dtype=np.int32)
+    for w in mem:
+        if 0 <= w < W and grads[w] is None:
+            raise ValueError("listed worker %d has no gradient buffer" % w)
+    out = np.empty(n, np.uint16 if out_dtype == "bf16" else np.float32)
+    rc = _load().oracle_group_reduce_f32(out.ctypes.data, DTYPE_BF16 if out_dtype == "bf16" else DTYPE_F32,
+                                         ptrs, W, dt, n, mem.ctypes.data, mem.shape[0],
+                                         SUM_ORDERS[sum_order])
+    if rc != 0:
+        raise ValueError("member list outside the definition (empty, duplicate or out-of-range member)")
+    return out
+
+
+def update_from_sums_f32(params, momentum, sums, n_reports, lr, mu, wd) -> None:
+    """One update from partial sums (float32 arrays, added left to right), the
+    mean taken over ``n_reports`` gradient reports; in place."""
+    n = params.shape[0]
+    for a in (params, momentum):
+        if a.dtype != np.float32 or a.shape != (n,) or not a.flags.c_contiguous or not a.flags.writeable:
+            raise ValueError("params/momentum must be contiguous writeable float32 of equal length")
+    R = len(sums)
+    ptrs = (ctypes.c_void_p * max(R, 1))()
+    for r, s in enumerate(sums):
+        if s.dtype != np.float32 or s.shape != (n,) or not s.flags.c_contiguous:
+            raise ValueError("partial sum %d must be contiguous float32 with %d elements" % (r, n))
+        ptrs[r] = s.ctypes.data
+    rc = _load().oracle_update_from_sums_f32(params.ctypes.data, momentum.ctypes.data, ptrs, R, n,
+                                             int(n_reports), float(np.float32(lr)), float(np.float32(mu)),
+                                             float(np.float32(wd)))
+    if rc != 0:
+        raise ValueError("need at least one partial sum and n_reports >= their number")
