@@ -33,7 +33,12 @@
  *     keeps no pointer after a call returns, except inside a caller-provided
  *     workspace.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t; NULL = legacy default
- *     stream) and the call returns without synchronizing.
+ *     stream) and the call returns without synchronizing.  The exceptions are
+ *     the calls that copy a table from ordinary host memory (star_multi_prepare,
+ *     star_multi_prepare_ex, star_group_update_multi_noalloc): such a copy
+ *     makes the host wait until earlier work on `cuda_stream` has finished and
+ *     the table is staged, and those calls refuse to run inside a stream
+ *     capture (STAR_ERR_UNSUPPORTED, nothing enqueued).
  *   - Every argument error is found on the host BEFORE anything is launched and
  *     leaves p and v untouched.  STAR_ERR_CUDA is a failed launch or runtime
  *     call; star_last_cuda_error() gives its cudaError_t.
@@ -41,9 +46,12 @@
  *     points return STAR_ERR_CUDA.
  *   - params, momentum and the scheduled gradient buffers must not overlap.
  *     Element-size alignment is required (4 bytes fp32, 2 bytes bf16).  Buffers
- *     aligned to 32 bytes take the full-width vector path; less aligned
- *     buffers take a narrower or element-by-element path with identical
- *     results (slower).
+ *     aligned to 32 bytes take the full-width vector path.  So do buffers that
+ *     are all views at one common element offset into 32-byte aligned storage
+ *     (the usual way a tensor ends up misaligned): up to 7 leading elements are
+ *     done one by one and the rest in vectors.  Buffers with no common
+ *     alignment phase take a narrower or element-by-element path (slower).
+ *     Results are identical on every path.
  */
 #ifndef STAR_H_
 #define STAR_H_
@@ -66,7 +74,7 @@ typedef enum {
     STAR_ERR_NULL_POINTER = 1,      /* a required pointer is NULL */
     STAR_ERR_INVALID_ARG = 2,       /* negative size, bad dtype, misaligned or overlapping buffers */
     STAR_ERR_BAD_SCHEDULE = 3,      /* empty group, duplicate or out-of-range member, bad offsets */
-    STAR_ERR_UNSUPPORTED = 4,       /* W above STAR_MAX_WORKERS */
+    STAR_ERR_UNSUPPORTED = 4,       /* W above STAR_MAX_WORKERS; a table-copying call inside a stream capture */
     STAR_ERR_WORKSPACE_TOO_SMALL = 5,
     STAR_ERR_CUDA = 6               /* see star_last_cuda_error() */
 } star_status_t;
@@ -221,9 +229,9 @@ STAR_API star_status_t star_group_update(float *params, float *momentum, const v
                                 int n_groups, float lr, float mu, float wd, void *cuda_stream);
 
 /* The same round with one learning rate per group, optional parameter
- * snapshots and a choice of the in-group summation order (sum_order; the tree
- * order keeps up to log2|G| partial sums per element in registers, runs at lower
- * occupancy and reaches about 65-75 % of the linear order's throughput).
+ * snapshots and a choice of the in-group summation order (sum_order; with
+ * groups of more than 4 members the tree order keeps partial sums per element
+ * in registers and runs at half the occupancy of the linear order).
  *   lrs        : host, n_groups learning rates.  Section IV-C1 ("Scaling learning
  *                rate after switching") sets the rate of an update built from y
  *                gradient reports to (y / N) x the SSGD rate; the caller computes
@@ -246,6 +254,47 @@ STAR_API star_status_t star_group_update_ex(float *params, float *momentum, cons
                                             star_sum_order_t sum_order, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
+ * All-reduce architecture (Section IV-B, paragraph "All-reduce architecture";
+ * Section IV-C1, Eq. 3).  Stragglers are taken out of the ring and report their
+ * gradients to a parent in the ring; the parent adds the gradients of the
+ * children that reported in time to its own, the ring sums its members'
+ * aggregates, and one update is made from the gradients of N - x + q workers.
+ * Two kernels cover the arithmetic of such a round on one GPU; moving the
+ * buffers between GPUs is the caller's (a collective library's) part, and
+ * every buffer handed to these calls is memory of the current device.
+ * ------------------------------------------------------------------------- */
+
+/* A parent's local aggregate: out[i] = g[m_0][i] + g[m_1][i] + ... over the
+ * `count` listed workers (own gradient first, then the children), each addition
+ * one binary32 operation, left to right or in tree order (sum_order), written as
+ * binary32 (out_dtype F32) or rounded to bf16, nearest even (BF16).
+ *   out     : device, n elements of out_dtype; must not overlap a listed buffer
+ *   grads   : host array of W device pointers (n elements of grad_dtype each);
+ *             only the listed entries are dereferenced
+ *   members : host, `count` distinct workers in [0, W); count == 0 is
+ *             STAR_ERR_BAD_SCHEDULE (an empty sum has no meaning in this round)
+ * n == 0 is a successful no-op.  One kernel launch; n * (count * sizeof(g) +
+ * sizeof(out)) bytes of traffic. */
+STAR_API star_status_t star_group_reduce(void *out, star_dtype_t out_dtype, const void *const *grads,
+                                         int W, star_dtype_t grad_dtype, int64_t n,
+                                         const int32_t *members, int count,
+                                         star_sum_order_t sum_order, void *cuda_stream);
+
+/* The one update of an all-reduce round from the R ring members' aggregates
+ * (binary32, n elements each, device), added left to right in the listed (ring)
+ * order; the mean divides by n_reports, the number of gradient reports behind
+ * the aggregates (N - x + q of Eq. 3, R <= n_reports <= 255):
+ *     s = sums[0][i] + sums[1][i] + ... ; gbar = s / n_reports ;
+ *     d = fma(wd, p, gbar) ; v = fma(mu, v, d) ; p = fma(-lr, v, p)
+ * sums: host array of R device pointers.  Every rank that applies this call to
+ * the same aggregates in the same order holds bit-identical parameters
+ * afterwards.  R == 0 with n_reports == 0, or n == 0, is a no-op.  One launch. */
+STAR_API star_status_t star_group_update_from_sums(float *params, float *momentum,
+                                                   const float *const *sums, int R, int64_t n,
+                                                   int n_reports, float lr, float mu, float wd,
+                                                   void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * Fused grouped update of a LIST of tensors (per-layer parameters) in one
  * launch.  The pointer table and tile map live in a caller-provided device
  * workspace that is prepared once per tensor list and reused every round.
@@ -264,10 +313,12 @@ typedef struct {
     int32_t W;
     int32_t grad_dtype;        /* star_dtype_t */
     int32_t tile_elements;     /* elements per tile */
+    int32_t n_snapshot_sets;   /* snapshot buffer sets registered by star_multi_prepare_ex (else 0) */
+    int32_t snapshot_dtype;    /* star_dtype_t of those buffers */
 } star_multi_plan_t;
 
 /* Bytes of device workspace needed for n_tensors tensors of the given sizes
- * (host array, elements per tensor, 0 allowed) and W workers. */
+ * (host array, elements per tensor, 0 allowed) and W workers (no snapshot sets). */
 STAR_API star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *sizes, int W,
                                          size_t *bytes_out);
 
@@ -278,8 +329,13 @@ STAR_API star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *
  * device, 256-byte aligned, at least star_multi_workspace_bytes() bytes.  The
  * table is built in ordinary host memory and copied with one cudaMemcpyAsync on
  * cuda_stream; the host copy is released before the call returns (a copy from
- * pageable memory returns once the data is staged), later work on the same
- * stream sees the table.  Not a per-round call: once per tensor list. */
+ * pageable memory returns once the data is staged, which makes the host wait
+ * for earlier work on cuda_stream), later work on the same stream sees the
+ * table.  Inside a stream capture the call returns STAR_ERR_UNSUPPORTED and
+ * enqueues nothing.  No buffer that a round writes (params, momentum) may
+ * share memory with any other buffer of the list, in the same or in another
+ * tensor (STAR_ERR_INVALID_ARG: e.g. a tied weight listed twice); gradient
+ * buffers may alias one another.  Not a per-round call: once per tensor list. */
 STAR_API star_status_t star_multi_prepare(int n_tensors, float *const *params, float *const *momentum,
                                  const void *const *grads, const int64_t *sizes, int W,
                                  star_dtype_t grad_dtype, void *d_workspace,
@@ -303,6 +359,42 @@ STAR_API star_status_t star_group_update_multi_lrs(const star_multi_plan_t *plan
                                                    const int32_t *group_members, int n_groups,
                                                    const float *lrs, float mu, float wd,
                                                    void *cuda_stream);
+
+/* Tensor lists with parameter snapshots and the tree order.  A snapshot SET is
+ * one buffer per tensor of the list; up to STAR_MAX_WORKERS sets are registered
+ * when the list is prepared (their pointers go into the same workspace table),
+ * and every round says which set, if any, receives the parameters as they stand
+ * right after each group's update -- the copy the server sends back to that
+ * group's workers (Section II) -- written in the same pass.
+ *   star_multi_workspace_bytes_ex : workspace size with n_snapshot_sets sets
+ *   star_multi_prepare_ex         : as star_multi_prepare, plus
+ *       snapshots      host array of n_tensors * n_snapshot_sets device pointers,
+ *                      entry [t * n_snapshot_sets + s] = tensor t's buffer of set
+ *                      s (sizes[t] elements of snapshot_dtype; NULL = tensor t is
+ *                      not captured by set s); snapshot buffers are written, so
+ *                      they must not overlap anything else in the list
+ *   star_group_update_multi_ex    : one round, one launch, with
+ *       lrs                    host, one learning rate per group (Section IV-C1)
+ *       snapshot_set_of_group  NULL, or host array of n_groups entries: the set
+ *                              (0 .. n_snapshot_sets-1) written after group k, or -1
+ *       sum_order              STAR_SUM_LINEAR or STAR_SUM_TREE (Section IV-D2b)
+ * Results equal star_group_update_ex applied to every tensor of the list. */
+STAR_API star_status_t star_multi_workspace_bytes_ex(int n_tensors, const int64_t *sizes, int W,
+                                                     int n_snapshot_sets, size_t *bytes_out);
+
+STAR_API star_status_t star_multi_prepare_ex(int n_tensors, float *const *params, float *const *momentum,
+                                             const void *const *grads, const int64_t *sizes, int W,
+                                             star_dtype_t grad_dtype, int n_snapshot_sets,
+                                             void *const *snapshots, star_dtype_t snapshot_dtype,
+                                             void *d_workspace, size_t workspace_bytes,
+                                             void *cuda_stream, star_multi_plan_t *plan_out);
+
+STAR_API star_status_t star_group_update_multi_ex(const star_multi_plan_t *plan,
+                                                  const int32_t *group_offsets,
+                                                  const int32_t *group_members, int n_groups,
+                                                  const float *lrs, float mu, float wd,
+                                                  const int32_t *snapshot_set_of_group,
+                                                  star_sum_order_t sum_order, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
  * Fused grouped update with the state and the gradients in HOST memory (the
@@ -365,7 +457,11 @@ STAR_API star_status_t star_group_update_host(float *h_params, float *h_momentum
  *     STAR_ERR_WORKSPACE_TOO_SMALL and nothing is launched.  1 MiB covers, for
  *     example, 292 tensors / 355 M elements / 16 workers (about 0.75 MiB).
  *   - The first call on each device looks up the array's device address (with
- *     that device current).  Make that first call outside any stream capture.
+ *     that device current).
+ *   - The call cannot be part of a stream capture, first call or not: the table
+ *     is copied from host memory that is released on return, which a captured
+ *     graph would read again at every replay.  When cuda_stream is capturing
+ *     the call returns STAR_ERR_UNSUPPORTED and enqueues nothing.
  *   - All calls on a device share the one array, and it keeps the previous
  *     call's table; each call rewrites the part it uses before its kernel
  *     reads it, so nothing has to start out zeroed.  Calls on one stream are
@@ -373,8 +469,10 @@ STAR_API star_status_t star_group_update_host(float *h_params, float *h_momentum
  *     without a dependency, or several host threads) race on the array: the
  *     caller must serialize them.
  *   - The table is rebuilt and copied (one cudaMemcpyAsync from pageable host
- *     memory) on every call; callers that can provide a workspace should
- *     prepare once and use star_group_update_multi.
+ *     memory) on every call.  That copy makes the host wait until the work
+ *     queued earlier on cuda_stream, the previous round included, has finished:
+ *     the call does not run ahead of the GPU.  Callers that can provide a
+ *     workspace should prepare once and use star_group_update_multi.
  * ------------------------------------------------------------------------- */
 #define STAR_STATIC_SCRATCH_BYTES (1u << 20)
 

@@ -56,6 +56,8 @@ class star_multi_plan_t(ctypes.Structure):
         ("W", ctypes.c_int32),
         ("grad_dtype", ctypes.c_int32),
         ("tile_elements", ctypes.c_int32),
+        ("n_snapshot_sets", ctypes.c_int32),
+        ("snapshot_dtype", ctypes.c_int32),
     ]
 
 
@@ -113,6 +115,17 @@ def _load() -> ctypes.CDLL:
     lib.star_group_update_multi_noalloc.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp, c_vp,
                                                     c_int, c_f, c_f, c_f, c_vp]
     lib.star_group_update_multi_noalloc.restype = c_int
+    lib.star_group_reduce.argtypes = [c_vp, c_int, c_vp, c_int, c_int, c_i64, c_vp, c_int, c_int, c_vp]
+    lib.star_group_reduce.restype = c_int
+    lib.star_group_update_from_sums.argtypes = [c_vp, c_vp, c_vp, c_int, c_i64, c_int, c_f, c_f, c_f, c_vp]
+    lib.star_group_update_from_sums.restype = c_int
+    lib.star_multi_workspace_bytes_ex.argtypes = [c_int, c_vp, c_int, c_int, c_vp]
+    lib.star_multi_workspace_bytes_ex.restype = c_int
+    lib.star_multi_prepare_ex.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_int, c_vp, c_int, c_vp,
+                                          ctypes.c_size_t, c_vp, c_vp]
+    lib.star_multi_prepare_ex.restype = c_int
+    lib.star_group_update_multi_ex.argtypes = [c_vp, c_vp, c_vp, c_int, c_vp, c_f, c_f, c_vp, c_int, c_vp]
+    lib.star_group_update_multi_ex.restype = c_int
     for name in ("star_schedule_validate", "star_schedule_static_x", "star_schedule_from_labels",
                  "star_schedule_dynamic_x", "star_group_update", "star_multi_workspace_bytes",
                  "star_multi_prepare", "star_group_update_multi"):
@@ -367,6 +380,53 @@ def star_group_update_ex(params: torch.Tensor, momentum: torch.Tensor,
                                      snap_arr, snap_dt, sum_order, _stream(stream)), "star_group_update_ex")
 
 
+def _grad_pointers(grads: Sequence[Optional[torch.Tensor]], n: int):
+    """(ctypes array of W device pointers, dtype code) of a list of flat gradient tensors."""
+    W = len(grads)
+    ptrs = (ctypes.c_void_p * max(W, 1))()
+    dt = None
+    for w, g in enumerate(grads):
+        if g is None:
+            continue
+        if not g.is_cuda or not g.is_contiguous() or g.numel() != n:
+            raise ValueError("gradient %d must be a contiguous CUDA tensor of %d elements" % (w, n))
+        d = _grad_dtype(g)
+        if dt is not None and d != dt:
+            raise TypeError("gradients differ in dtype")
+        dt = d
+        ptrs[w] = g.data_ptr()
+    return ptrs, STAR_DTYPE_F32 if dt is None else dt
+
+
+def star_group_reduce(out: torch.Tensor, grads: Sequence[Optional[torch.Tensor]], members: Sequence[int],
+                      sum_order: int = STAR_SUM_LINEAR, stream=None) -> None:
+    """``out[i] = grads[members[0]][i] + grads[members[1]][i] + ...`` (what a parent
+    of the all-reduce architecture forwards to the ring); ``out`` is a float32
+    or bfloat16 CUDA tensor."""
+    n = out.numel()
+    if not out.is_cuda or not out.is_contiguous():
+        raise TypeError("out must be a contiguous CUDA tensor")
+    ptrs, dt = _grad_pointers(grads, n)
+    _check(_lib.star_group_reduce(out.data_ptr(), _grad_dtype(out), ptrs, len(grads), dt, n, _i32(members),
+                                  len(members), sum_order, _stream(stream)), "star_group_reduce")
+
+
+def star_group_update_from_sums(params: torch.Tensor, momentum: torch.Tensor, sums: Sequence[torch.Tensor],
+                                n_reports: int, lr: float, mu: float, wd: float, stream=None) -> None:
+    """One update from the ring members' aggregates ``sums`` (float32 CUDA tensors,
+    added in the listed order), the mean taken over ``n_reports`` gradient reports."""
+    n = params.numel()
+    p, v = _state(params, "params"), _state(momentum, "momentum")
+    if momentum.numel() != n:
+        raise ValueError("params and momentum differ in size")
+    for r, t in enumerate(sums):
+        if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or t.numel() != n:
+            raise ValueError("sum %d must be a contiguous float32 CUDA tensor of %d elements" % (r, n))
+    ptrs = (ctypes.c_void_p * max(len(sums), 1))(*[t.data_ptr() for t in sums])
+    _check(_lib.star_group_update_from_sums(p, v, ptrs, len(sums), n, n_reports, lr, mu, wd, _stream(stream)),
+           "star_group_update_from_sums")
+
+
 def star_multi_workspace_bytes(sizes: Sequence[int], W: int) -> int:
     out = ctypes.c_size_t(0)
     arr = (ctypes.c_int64 * max(len(sizes), 1))(*sizes)
@@ -431,6 +491,89 @@ def star_group_update_multi_lrs(plan: star_multi_plan_t, group_offsets: Sequence
     _check(_lib.star_group_update_multi_lrs(ctypes.byref(plan), _i32(group_offsets), _i32(group_members), K,
                                             (ctypes.c_float * max(K, 1))(*lrs), mu, wd, _stream(stream)),
            "star_group_update_multi_lrs")
+
+
+def star_multi_workspace_bytes_ex(sizes: Sequence[int], W: int, n_snapshot_sets: int) -> int:
+    out = ctypes.c_size_t(0)
+    arr = (ctypes.c_int64 * max(len(sizes), 1))(*sizes)
+    _check(_lib.star_multi_workspace_bytes_ex(len(sizes), arr, W, n_snapshot_sets, ctypes.byref(out)),
+           "star_multi_workspace_bytes_ex")
+    return out.value
+
+
+def _list_pointers(params, momentum, grads):
+    """Pointer arrays (P, V, G, sizes array, dtype code) of a tensor list;
+    ``grads[w][t]`` = worker w's gradient for tensor t."""
+    T, W = len(params), len(grads)
+    if len(momentum) != T or any(len(g) != T for g in grads):
+        raise ValueError("params, momentum and every worker's gradient list need one entry per tensor")
+    sizes = [p.numel() for p in params]
+    if any(v.numel() != s for v, s in zip(momentum, sizes)):
+        raise ValueError("params and momentum differ in size")
+    P = (ctypes.c_void_p * max(T, 1))(*[_state(p, "params") if p.numel() else None for p in params])
+    V = (ctypes.c_void_p * max(T, 1))(*[_state(v, "momentum") if v.numel() else None for v in momentum])
+    G = (ctypes.c_void_p * max(T * W, 1))()
+    dt = None
+    for w in range(W):
+        for t in range(T):
+            g = grads[w][t]
+            if g is None or sizes[t] == 0:
+                continue
+            if not g.is_cuda or not g.is_contiguous() or g.numel() != sizes[t]:
+                raise ValueError("gradient [%d][%d] must be a contiguous CUDA tensor of %d elements"
+                                 % (w, t, sizes[t]))
+            d = _grad_dtype(g)
+            if dt is not None and d != dt:
+                raise TypeError("gradients differ in dtype")
+            dt = d
+            G[t * W + w] = g.data_ptr()
+    S = (ctypes.c_int64 * max(T, 1))(*sizes)
+    return P, V, G, S, sizes, STAR_DTYPE_F32 if dt is None else dt
+
+
+def star_multi_prepare_ex(params: Sequence[torch.Tensor], momentum: Sequence[torch.Tensor],
+                          grads: Sequence[Sequence[Optional[torch.Tensor]]],
+                          snapshot_sets: Sequence[Sequence[Optional[torch.Tensor]]], workspace: torch.Tensor,
+                          stream=None) -> star_multi_plan_t:
+    """As :func:`star_multi_prepare`, registering ``snapshot_sets[s][t]`` (tensor
+    t's buffer of snapshot set s, all float32 or all bfloat16, or None)."""
+    T, W, S_sets = len(params), len(grads), len(snapshot_sets)
+    P, V, G, S, sizes, dt = _list_pointers(params, momentum, grads)
+    if any(len(one) != T for one in snapshot_sets):
+        raise ValueError("every snapshot set needs one entry (tensor or None) per tensor")
+    snaps = (ctypes.c_void_p * max(T * S_sets, 1))()
+    kinds = set()
+    for s_index, one in enumerate(snapshot_sets):
+        for t, buf in enumerate(one):
+            if buf is None or sizes[t] == 0:
+                continue
+            if not buf.is_cuda or not buf.is_contiguous() or buf.numel() != sizes[t]:
+                raise ValueError("snapshot [%d][%d] must be a contiguous CUDA tensor of %d elements"
+                                 % (s_index, t, sizes[t]))
+            kinds.add(_grad_dtype(buf))
+            snaps[t * S_sets + s_index] = buf.data_ptr()
+    if len(kinds) > 1:
+        raise TypeError("snapshots differ in dtype")
+    if workspace.dtype != torch.uint8 or not workspace.is_cuda or not workspace.is_contiguous():
+        raise TypeError("workspace must be a contiguous uint8 CUDA tensor")
+    plan = star_multi_plan_t()
+    _check(_lib.star_multi_prepare_ex(T, P, V, G, S, W, dt, S_sets, snaps, kinds.pop() if kinds else STAR_DTYPE_F32,
+                                      workspace.data_ptr(), workspace.numel(), _stream(stream),
+                                      ctypes.byref(plan)), "star_multi_prepare_ex")
+    return plan
+
+
+def star_group_update_multi_ex(plan: star_multi_plan_t, group_offsets: Sequence[int],
+                               group_members: Sequence[int], lrs: Sequence[float], mu: float, wd: float,
+                               snapshot_set_of_group: Optional[Sequence[int]] = None,
+                               sum_order: int = STAR_SUM_LINEAR, stream=None) -> None:
+    K = len(group_offsets) - 1 if len(group_offsets) else 0
+    if len(lrs) != K or (snapshot_set_of_group is not None and len(snapshot_set_of_group) != K):
+        raise ValueError("need one learning rate (and one snapshot set index) per group")
+    sets = None if snapshot_set_of_group is None else _i32(snapshot_set_of_group)
+    _check(_lib.star_group_update_multi_ex(ctypes.byref(plan), _i32(group_offsets), _i32(group_members), K,
+                                           (ctypes.c_float * max(K, 1))(*lrs), mu, wd, sets, sum_order,
+                                           _stream(stream)), "star_group_update_multi_ex")
 
 
 def star_host_workspace_bytes(max_scheduled: int, grad_dtype: torch.dtype, chunk_elements: int) -> int:

@@ -91,8 +91,8 @@ star_status_t flatten_schedule(const int32_t *group_offsets, const int32_t *grou
         const int first = group_offsets[k], last = group_offsets[k + 1];
         for (int j = first; j < last; ++j) {
             out->member[j] = static_cast<uint8_t>(group_members[j]);
-            out->index_in_group[j] = static_cast<uint8_t>(j - first);
         }
+        out->size_at_start[first] = static_cast<uint8_t>(last - first);
         out->group_size[last - 1] = static_cast<uint8_t>(last - first);
         out->neg_lr[last - 1] = lrs ? -lrs[k] : -lr;
     }
@@ -113,37 +113,68 @@ bool aligned(const void *p, size_t bytes) { return reinterpret_cast<uintptr_t>(p
 constexpr int kVecBF16 = 8;
 constexpr int kVecF32 = 4;
 constexpr int kDepthVector = 4;
-constexpr int kDepthScalar = 4;
 constexpr int kDepthNarrow = 8;           // flat kernels whose gradient loads are narrower than 16 bytes
-constexpr int kDepthTree = 2;             // tree order with 4 or 6 levels: registers go to the pending partial sums
 constexpr int kVecBF16Half = 4;           // bf16 with buffers aligned for 16-byte state / 8-byte gradient accesses
 
-// Alignment of the buffers of a call: the smallest power of two (capped at 32)
-// that divides every state (p, v, snapshot) address, and every gradient address.
-struct Alignment {
-    unsigned state = 32, grad = 32;
-    static unsigned of(const void *p)
-    {
-        const uintptr_t a = reinterpret_cast<uintptr_t>(p);
-        unsigned k = 32;
-        while (k > 1 && a % k != 0) k /= 2;
-        return k;
-    }
-    void add_state(const void *p) { state = std::min(state, of(p)); }
-    void add_grad(const void *p) { grad = std::min(grad, of(p)); }
+// The device buffers one thread's vector touches (of a call, or of one tensor
+// of a list), with their element sizes.
+struct Buffers {
+    struct Item {
+        uintptr_t addr;
+        unsigned elem;
+    };
+    Item item[2 + 2 * kMaxWorkers];
+    int count = 0;
+    void add(const void *p, unsigned elem) { item[count++] = Item{reinterpret_cast<uintptr_t>(p), elem}; }
 };
 
-// Elements per thread the alignment allows.  bf16: 8 (32-byte state accesses,
-// 16-byte gradient loads) or 4 (16 / 8 bytes); fp32: 4 (16-byte accesses); else
-// the element-by-element kernel.
-int vector_width(star_dtype_t dt, const Alignment &al)
+// Elements per thread and the number of leading elements in front of the
+// vector body.  A vector of `vec` elements needs every buffer aligned to vec
+// elements of its own type (bf16, vec 8: 32 bytes for fp32 state, 16 bytes for
+// gradients) at the element where the body starts.  Buffers that are views at
+// one common element offset into aligned storage reach that alignment together
+// after `head` < vec elements, which are then done one by one; buffers with no
+// common phase fall back to a narrower vector (bf16 flat kernels: 4) or to the
+// element-by-element kernel (vec 1).  Results do not depend on the choice.
+struct VectorPlan {
+    int vec = 1;
+    int head = 0;
+};
+
+VectorPlan plan_vector(star_dtype_t dt, const Buffers &b, int64_t n, bool allow_half)
 {
-    if (dt == STAR_DTYPE_BF16) {
-        if (al.state >= 32 && al.grad >= 16) return kVecBF16;
-        if (al.state >= 16 && al.grad >= 8) return kVecBF16Half;
-        return 1;
+    const int candidates[2] = {dt == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32,
+                               dt == STAR_DTYPE_BF16 && allow_half ? kVecBF16Half : 0};
+    for (int vec : candidates) {
+        if (vec <= 1 || b.count == 0) continue;
+        const Buffers::Item &f = b.item[0];
+        const unsigned span = f.elem * static_cast<unsigned>(vec);
+        const unsigned r = static_cast<unsigned>(f.addr % span);
+        const int head = r == 0 ? 0 : static_cast<int>((span - r) / f.elem);
+        bool ok = true;
+        for (int i = 0; i < b.count && ok; ++i) {
+            const Buffers::Item &x = b.item[i];
+            ok = (x.addr + static_cast<uintptr_t>(head) * x.elem) % (x.elem * static_cast<unsigned>(vec)) == 0;
+        }
+        if (ok && n >= head + vec) return VectorPlan{vec, head};
     }
-    return al.state >= 16 && al.grad >= 16 ? kVecF32 : 1;
+    return VectorPlan{};
+}
+
+// Launch of a grid-stride kernel over n_vec vectors of one flat tensor.
+template <typename Kernel, typename Args>
+star_status_t launch_grid_stride(Kernel kernel, Geometry *cache, const Args &args, int64_t n_vec, cudaStream_t stream)
+{
+    int blocks = 0;
+    cudaError_t e = resident_blocks(kernel, cache, &blocks);
+    if (e != cudaSuccess) return cuda_failed(e);
+    const int64_t work = (n_vec + kBlockThreads - 1) / kBlockThreads;
+    const int grid = choose_grid(work, blocks);
+    kernel<<<grid, kBlockThreads, 0, stream>>>(args);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return STAR_OK;
 }
 
 template <typename G, int VEC>
@@ -152,17 +183,7 @@ star_status_t launch_flat(const FlatArgs &args, cudaStream_t stream)
     static Geometry cache[kMaxDevices];
     // Narrow loads (element by element, half-width bf16) keep more of them in flight.
     constexpr int depth = VEC * G::kBytes >= 16 ? kDepthVector : kDepthNarrow;
-    auto kernel = star_update_flat_kernel<G, VEC, depth>;
-    int blocks = 0;
-    cudaError_t e = resident_blocks(kernel, cache, &blocks);
-    if (e != cudaSuccess) return cuda_failed(e);
-    const int64_t work = (args.n / VEC + kBlockThreads - 1) / kBlockThreads;
-    const int grid = choose_grid(work, blocks);
-    kernel<<<grid, kBlockThreads, 0, stream>>>(args);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_failed(e);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return STAR_OK;
+    return launch_grid_stride(star_update_flat_kernel<G, VEC, depth>, cache, args, (args.n - args.head) / VEC, stream);
 }
 
 }  // namespace
@@ -189,11 +210,11 @@ namespace {
 
 // Everything the flat entry points check before a launch.  On STAR_OK either
 // *noop is set (empty tensor or empty schedule: nothing to do) or *args is
-// complete and *align holds the alignment of its buffers.
+// complete (but for args->head) and *buffers lists the buffers of the call.
 star_status_t prepare_flat(float *params, float *momentum, const void *const *grads, int W,
                            star_dtype_t grad_dtype, int64_t n, const int32_t *group_offsets,
                            const int32_t *group_members, int n_groups, float lr, const float *lrs, float mu,
-                           float wd, FlatArgs *args, Alignment *align, bool *noop)
+                           float wd, FlatArgs *args, Buffers *buffers, bool *noop)
 {
     *noop = false;
     if (n < 0 || W < 0) return STAR_ERR_INVALID_ARG;
@@ -206,12 +227,12 @@ star_status_t prepare_flat(float *params, float *momentum, const void *const *gr
         return STAR_OK;
     }
     if (!params || !momentum || !grads) return STAR_ERR_NULL_POINTER;
-    const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const unsigned gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
     const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
     if (!aligned(params, 4) || !aligned(momentum, 4)) return STAR_ERR_INVALID_ARG;
     if (overlaps(params, state_bytes, momentum, state_bytes)) return STAR_ERR_INVALID_ARG;
-    align->add_state(params);
-    align->add_state(momentum);
+    buffers->add(params, 4);
+    buffers->add(momentum, 4);
     std::memset(args->grads, 0, sizeof args->grads);
     for (int j = 0; j < args->sched.n_slots; ++j) {
         const int w = args->sched.member[j];
@@ -220,51 +241,58 @@ star_status_t prepare_flat(float *params, float *momentum, const void *const *gr
         if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
         if (overlaps(g, grad_bytes, params, state_bytes) || overlaps(g, grad_bytes, momentum, state_bytes))
             return STAR_ERR_INVALID_ARG;
-        align->add_grad(g);
+        buffers->add(g, gsize);
         args->grads[w] = g;
     }
     args->params = params;
     args->momentum = momentum;
     args->n = n;
+    args->head = 0;
     args->hyper = Hyper{mu, wd};
     return STAR_OK;
 }
 
-star_status_t dispatch_flat(const FlatArgs &args, star_dtype_t grad_dtype, const Alignment &align,
-                            cudaStream_t stream)
+star_status_t dispatch_flat(FlatArgs &args, star_dtype_t grad_dtype, const VectorPlan &plan, cudaStream_t stream)
 {
-    const int vec = vector_width(grad_dtype, align);
+    args.head = plan.head;
     if (grad_dtype == STAR_DTYPE_BF16) {
-        if (vec == kVecBF16) return launch_flat<GradBF16, kVecBF16>(args, stream);
-        if (vec == kVecBF16Half) return launch_flat<GradBF16, kVecBF16Half>(args, stream);
+        if (plan.vec == kVecBF16) return launch_flat<GradBF16, kVecBF16>(args, stream);
+        if (plan.vec == kVecBF16Half) return launch_flat<GradBF16, kVecBF16Half>(args, stream);
         return launch_flat<GradBF16, 1>(args, stream);
     }
-    return vec == kVecF32 ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
+    return plan.vec == kVecF32 ? launch_flat<GradF32, kVecF32>(args, stream) : launch_flat<GradF32, 1>(args, stream);
 }
 
 template <typename G, int VEC, int TREE>
 star_status_t launch_flat_snapshot(const SnapshotArgs &args, cudaStream_t stream)
 {
     static Geometry cache[kMaxDevices];
-    constexpr int depth = VEC == 1 ? kDepthScalar : (TREE > 2 ? kDepthTree : kDepthVector);
-    auto kernel = star_update_flat_snapshot_kernel<G, VEC, depth, TREE>;
-    int blocks = 0;
-    cudaError_t e = resident_blocks(kernel, cache, &blocks);
-    if (e != cudaSuccess) return cuda_failed(e);
-    const int64_t work = (args.flat.n / VEC + kBlockThreads - 1) / kBlockThreads;
-    const int grid = choose_grid(work, blocks);
-    kernel<<<grid, kBlockThreads, 0, stream>>>(args);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_failed(e);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return STAR_OK;
+    return launch_grid_stride(star_update_flat_snapshot_kernel<G, VEC, kDepthVector, TREE>, cache, args,
+                              (args.flat.n - args.flat.head) / VEC, stream);
 }
 
 // The extended kernels come in the full vector width and element by element only.
 template <typename G, int VEC, int TREE>
-star_status_t dispatch_snapshot(const SnapshotArgs &args, bool vector_ok, cudaStream_t stream)
+star_status_t dispatch_snapshot(SnapshotArgs &args, const VectorPlan &plan, cudaStream_t stream)
 {
-    return vector_ok ? launch_flat_snapshot<G, VEC, TREE>(args, stream) : launch_flat_snapshot<G, 1, TREE>(args, stream);
+    args.flat.head = plan.head;
+    return plan.vec == VEC ? launch_flat_snapshot<G, VEC, TREE>(args, stream)
+                           : launch_flat_snapshot<G, 1, TREE>(args, stream);
+}
+
+// Span of the tree-order kernel that serves groups of up to `largest` members
+// (0: the linear kernel; up to two members both orders are the same sum).
+int tree_span(star_sum_order_t order, int largest)
+{
+    if (order != STAR_SUM_TREE || largest <= 2) return 0;
+    return largest <= 4 ? 4 : largest <= 16 ? 16 : 64;
+}
+
+int largest_group(const int32_t *group_offsets, int n_groups)
+{
+    int largest = 1;
+    for (int k = 0; k < n_groups; ++k) largest = std::max(largest, group_offsets[k + 1] - group_offsets[k]);
+    return largest;
 }
 
 }  // namespace
@@ -275,12 +303,13 @@ extern "C" star_status_t star_group_update(float *params, float *momentum, const
                                            int n_groups, float lr, float mu, float wd, void *cuda_stream)
 {
     FlatArgs args;
-    Alignment align;
+    Buffers buffers;
     bool noop = false;
     const star_status_t st = prepare_flat(params, momentum, grads, W, grad_dtype, n, group_offsets, group_members,
-                                          n_groups, lr, nullptr, mu, wd, &args, &align, &noop);
+                                          n_groups, lr, nullptr, mu, wd, &args, &buffers, &noop);
     if (st != STAR_OK || noop) return st;
-    return dispatch_flat(args, grad_dtype, align, static_cast<cudaStream_t>(cuda_stream));
+    return dispatch_flat(args, grad_dtype, plan_vector(grad_dtype, buffers, n, true),
+                         static_cast<cudaStream_t>(cuda_stream));
 }
 
 // Per-group learning rates and parameter snapshots.
@@ -296,17 +325,17 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
     if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
     SnapshotArgs sargs;
     FlatArgs &args = sargs.flat;
-    Alignment align;
+    Buffers buffers;
     bool noop = false;
     const star_status_t st = prepare_flat(params, momentum, grads, W, grad_dtype, n, group_offsets, group_members,
-                                          n_groups, 0.0f, lrs, mu, wd, &args, &align, &noop);
+                                          n_groups, 0.0f, lrs, mu, wd, &args, &buffers, &noop);
     if (st != STAR_OK || noop) return st;
 
     const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
     const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
     std::memset(sargs.snapshots, 0, sizeof sargs.snapshots);
     sargs.snapshot_bf16 = snapshot_dtype == STAR_DTYPE_BF16 ? 1 : 0;
-    const size_t snap_elem = snapshot_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const unsigned snap_elem = snapshot_dtype == STAR_DTYPE_BF16 ? 2 : 4;
     const size_t snap_bytes = static_cast<size_t>(n) * snap_elem;
     bool any_snapshot = false;
     for (int k = 0; snapshots && k < n_groups; ++k) {
@@ -319,28 +348,123 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
             if (overlaps(snap, snap_bytes, args.grads[args.sched.member[j]], grad_bytes)) return STAR_ERR_INVALID_ARG;
         for (int l = 0; l < k; ++l)
             if (snapshots[l] && overlaps(snap, snap_bytes, snapshots[l], snap_bytes)) return STAR_ERR_INVALID_ARG;
-        // a bf16 snapshot moves half the bytes: 16-byte alignment serves the full vector width
-        if (snapshot_dtype == STAR_DTYPE_BF16) align.state = std::min(align.state, 2 * Alignment::of(snap));
-        else align.add_state(snap);
+        buffers.add(snap, snap_elem);
         sargs.snapshots[group_offsets[k + 1] - 1] = snap;
         any_snapshot = true;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const bool vector_ok = vector_width(grad_dtype, align) == (grad_dtype == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32);
-    int largest_group = 1;
-    for (int k = 0; k < n_groups; ++k) largest_group = std::max(largest_group, group_offsets[k + 1] - group_offsets[k]);
-    if (sum_order == STAR_SUM_TREE && largest_group > 2) {      // up to two members both orders are the same sum
-        const bool bf16 = grad_dtype == STAR_DTYPE_BF16;
-        if (largest_group <= 4) return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 2>(sargs, vector_ok, stream)
-                                            : dispatch_snapshot<GradF32, kVecF32, 2>(sargs, vector_ok, stream);
-        if (largest_group <= 16) return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 4>(sargs, vector_ok, stream)
-                                             : dispatch_snapshot<GradF32, kVecF32, 4>(sargs, vector_ok, stream);
-        return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 6>(sargs, vector_ok, stream)
-                    : dispatch_snapshot<GradF32, kVecF32, 6>(sargs, vector_ok, stream);
+    const int tree = tree_span(sum_order, largest_group(group_offsets, n_groups));
+    if (tree == 0 && !any_snapshot)        // per-group rates only
+        return dispatch_flat(args, grad_dtype, plan_vector(grad_dtype, buffers, n, true), stream);
+    const VectorPlan plan = plan_vector(grad_dtype, buffers, n, false);
+    const bool bf16 = grad_dtype == STAR_DTYPE_BF16;
+    switch (tree) {
+    case 4: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 4>(sargs, plan, stream)
+                        : dispatch_snapshot<GradF32, kVecF32, 4>(sargs, plan, stream);
+    case 16: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 16>(sargs, plan, stream)
+                         : dispatch_snapshot<GradF32, kVecF32, 16>(sargs, plan, stream);
+    case 64: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 64>(sargs, plan, stream)
+                         : dispatch_snapshot<GradF32, kVecF32, 64>(sargs, plan, stream);
+    default: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 0>(sargs, plan, stream)
+                         : dispatch_snapshot<GradF32, kVecF32, 0>(sargs, plan, stream);
     }
-    if (!any_snapshot) return dispatch_flat(args, grad_dtype, align, stream);   // per-group rates only
-    return grad_dtype == STAR_DTYPE_BF16 ? dispatch_snapshot<GradBF16, kVecBF16, 0>(sargs, vector_ok, stream)
-                                         : dispatch_snapshot<GradF32, kVecF32, 0>(sargs, vector_ok, stream);
+}
+
+// ---------------------------------------------------------------------------
+// All-reduce architecture: a parent's local sum, and the update from the ring
+// members' sums.
+// ---------------------------------------------------------------------------
+namespace {
+
+template <typename G, int VEC, int TREE>
+star_status_t launch_reduce(const ReduceArgs &args, cudaStream_t stream)
+{
+    static Geometry cache[kMaxDevices];
+    constexpr int depth = VEC * G::kBytes >= 16 ? kDepthVector : kDepthNarrow;
+    return launch_grid_stride(star_group_reduce_kernel<G, VEC, depth, TREE>, cache, args,
+                              (args.n - args.head) / VEC, stream);
+}
+
+template <typename G, int VEC>
+star_status_t dispatch_reduce(ReduceArgs &args, const VectorPlan &plan, int tree, cudaStream_t stream)
+{
+    args.head = plan.head;
+    const bool vec = plan.vec == VEC;
+    switch (tree) {
+    case 4: return vec ? launch_reduce<G, VEC, 4>(args, stream) : launch_reduce<G, 1, 4>(args, stream);
+    case 16: return vec ? launch_reduce<G, VEC, 16>(args, stream) : launch_reduce<G, 1, 16>(args, stream);
+    case 64: return vec ? launch_reduce<G, VEC, 64>(args, stream) : launch_reduce<G, 1, 64>(args, stream);
+    default: return vec ? launch_reduce<G, VEC, 0>(args, stream) : launch_reduce<G, 1, 0>(args, stream);
+    }
+}
+
+}  // namespace
+
+extern "C" star_status_t star_group_reduce(void *out, star_dtype_t out_dtype, const void *const *grads, int W,
+                                           star_dtype_t grad_dtype, int64_t n, const int32_t *members,
+                                           int count, star_sum_order_t sum_order, void *cuda_stream)
+{
+    if (n < 0 || W < 0 || count < 0) return STAR_ERR_INVALID_ARG;
+    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (out_dtype != STAR_DTYPE_F32 && out_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (sum_order != STAR_SUM_LINEAR && sum_order != STAR_SUM_TREE) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    if (count == 0) return STAR_ERR_BAD_SCHEDULE;           // the sum of nothing is not defined here
+    if (!members) return STAR_ERR_NULL_POINTER;
+    const int32_t one_group[2] = {0, count};
+    const star_status_t st = star_schedule_validate(one_group, members, 1, W);
+    if (st != STAR_OK) return st;
+    if (n == 0) return STAR_OK;
+    if (!out || !grads) return STAR_ERR_NULL_POINTER;
+
+    const unsigned gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4, osize = out_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const size_t grad_bytes = static_cast<size_t>(n) * gsize, out_bytes = static_cast<size_t>(n) * osize;
+    if (!aligned(out, osize)) return STAR_ERR_INVALID_ARG;
+    ReduceArgs args;
+    std::memset(&args, 0, sizeof args);
+    Buffers buffers;
+    buffers.add(out, osize);
+    for (int j = 0; j < count; ++j) {
+        const void *g = grads[members[j]];
+        if (!g) return STAR_ERR_NULL_POINTER;
+        if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
+        if (overlaps(g, grad_bytes, out, out_bytes)) return STAR_ERR_INVALID_ARG;
+        buffers.add(g, gsize);
+        args.src[j] = g;
+    }
+    args.out = out;
+    args.n = n;
+    args.count = count;
+    args.out_bf16 = out_dtype == STAR_DTYPE_BF16 ? 1 : 0;
+    const VectorPlan plan = plan_vector(grad_dtype, buffers, n, false);
+    const int tree = tree_span(sum_order, count);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    return grad_dtype == STAR_DTYPE_BF16 ? dispatch_reduce<GradBF16, kVecBF16>(args, plan, tree, stream)
+                                         : dispatch_reduce<GradF32, kVecF32>(args, plan, tree, stream);
+}
+
+extern "C" star_status_t star_group_update_from_sums(float *params, float *momentum, const float *const *sums,
+                                                     int R, int64_t n, int n_reports, float lr, float mu,
+                                                     float wd, void *cuda_stream)
+{
+    if (R < 0 || n < 0) return STAR_ERR_INVALID_ARG;
+    if (R > STAR_MAX_WORKERS || n_reports > 255) return STAR_ERR_UNSUPPORTED;
+    if (R == 0) return n_reports == 0 ? STAR_OK : STAR_ERR_INVALID_ARG;
+    if (n_reports < R) return STAR_ERR_INVALID_ARG;
+    int32_t members[STAR_MAX_WORKERS];
+    for (int r = 0; r < R; ++r) members[r] = r;
+    const int32_t one_group[2] = {0, R};
+    FlatArgs args;
+    Buffers buffers;
+    bool noop = false;
+    const star_status_t st =
+        prepare_flat(params, momentum, reinterpret_cast<const void *const *>(sums), R, STAR_DTYPE_F32, n, one_group,
+                     members, 1, lr, nullptr, mu, wd, &args, &buffers, &noop);
+    if (st != STAR_OK || noop) return st;
+    // The mean is taken over the gradient reports behind the sums, not over the sums.
+    args.sched.group_size[R - 1] = static_cast<uint8_t>(n_reports);
+    return dispatch_flat(args, STAR_DTYPE_F32, plan_vector(STAR_DTYPE_F32, buffers, n, false),
+                         static_cast<cudaStream_t>(cuda_stream));
 }
 
 // ---------------------------------------------------------------------------
@@ -354,22 +478,24 @@ constexpr int64_t tile_elements(star_dtype_t dt)
 }
 
 // The workspace is sized for the smaller (fp32) tile, i.e. the larger tile
-// count, so that its size does not depend on the gradient dtype.
+// count, so that its size does not depend on the gradient dtype, plus one tile
+// per tensor for leading elements in front of a vector-aligned body.
 constexpr int64_t kTileForSizing = static_cast<int64_t>(kBlockThreads) * kVecF32;
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t tensors_off, grads_off, tiles_off, total;
+    size_t tensors_off, grads_off, snaps_off, tiles_off, total;
 };
 
-WorkspaceLayout layout_for(int n_tensors, int W, int64_t n_tiles)
+WorkspaceLayout layout_for(int n_tensors, int W, int n_sets, int64_t n_tiles)
 {
+    const size_t T = static_cast<size_t>(n_tensors);
     WorkspaceLayout l;
     l.tensors_off = 0;
-    l.grads_off = round_up(l.tensors_off + sizeof(TensorEntry) * static_cast<size_t>(n_tensors), kWorkspaceAlign);
-    l.tiles_off = round_up(l.grads_off + sizeof(void *) * static_cast<size_t>(n_tensors) * static_cast<size_t>(W),
-                           kWorkspaceAlign);
+    l.grads_off = round_up(l.tensors_off + sizeof(TensorEntry) * T, kWorkspaceAlign);
+    l.snaps_off = round_up(l.grads_off + sizeof(void *) * T * static_cast<size_t>(W), kWorkspaceAlign);
+    l.tiles_off = round_up(l.snaps_off + sizeof(void *) * T * static_cast<size_t>(n_sets), kWorkspaceAlign);
     l.total = round_up(l.tiles_off + sizeof(int32_t) * static_cast<size_t>(n_tiles), kWorkspaceAlign);
     if (l.total == 0) l.total = kWorkspaceAlign;
     return l;
@@ -381,75 +507,79 @@ star_status_t count_tiles(int n_tensors, const int64_t *sizes, int64_t tile, int
     *total = 0;
     for (int t = 0; t < n_tensors; ++t) {
         if (sizes[t] < 0) return STAR_ERR_INVALID_ARG;
-        *n_tiles += (sizes[t] + tile - 1) / tile;
+        *n_tiles += (sizes[t] + tile - 1) / tile + (sizes[t] > 0 ? 1 : 0);
         *total += sizes[t];
     }
     return STAR_OK;
 }
 
-template <typename G, int VEC>
-star_status_t launch_multi(const MultiArgs &args, cudaStream_t stream)
+// No buffer that the round writes (p, v, snapshots) may share memory with any
+// other buffer of the list: different blocks update different tensors at the
+// same time.  Gradients are only read and may alias one another.
+struct Interval {
+    uintptr_t begin, end;
+    bool written;
+};
+
+bool written_buffers_are_disjoint(std::vector<Interval> &iv)
 {
-    static Geometry cache[kMaxDevices];
-    auto kernel = star_update_multi_kernel<G, VEC, kDepthVector>;
-    int blocks = 0;
-    cudaError_t e = resident_blocks(kernel, cache, &blocks);
-    if (e != cudaSuccess) return cuda_failed(e);
-    // The tile-map kernel pays a table lookup per block: measured on B200 the
-    // persistent grid is the faster shape for it at every list size tried.
-    const int grid = static_cast<int>(args.n_tiles < blocks ? args.n_tiles : blocks);
-    kernel<<<grid, kBlockThreads, 0, stream>>>(args);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_failed(e);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return STAR_OK;
+    std::sort(iv.begin(), iv.end(), [](const Interval &a, const Interval &b) { return a.begin < b.begin; });
+    uintptr_t end_any = 0, end_written = 0;
+    for (const Interval &x : iv) {
+        if (x.begin < (x.written ? end_any : end_written)) return false;
+        end_any = std::max(end_any, x.end);
+        if (x.written) end_written = std::max(end_written, x.end);
+    }
+    return true;
 }
 
-}  // namespace
-
-extern "C" star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *sizes, int W,
-                                                    size_t *bytes_out)
+// The prepare calls copy from a host buffer that is released on return: inside
+// a stream capture that copy would be replayed from freed memory.
+star_status_t refuse_capture(cudaStream_t stream)
 {
-    if (!bytes_out) return STAR_ERR_NULL_POINTER;
-    if (n_tensors < 0 || W < 0) return STAR_ERR_INVALID_ARG;
-    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
-    if (n_tensors > 0 && !sizes) return STAR_ERR_NULL_POINTER;
-    int64_t n_tiles = 0, total = 0;
-    const star_status_t st = count_tiles(n_tensors, sizes, kTileForSizing, &n_tiles, &total);
-    if (st != STAR_OK) return st;
-    *bytes_out = layout_for(n_tensors, W, n_tiles).total;
-    return STAR_OK;
+    cudaStreamCaptureStatus status = cudaStreamCaptureStatusNone;
+    const cudaError_t e = cudaStreamIsCapturing(stream, &status);
+    if (e != cudaSuccess) return cuda_failed(e);
+    return status == cudaStreamCaptureStatusNone ? STAR_OK : STAR_ERR_UNSUPPORTED;
 }
 
-extern "C" star_status_t star_multi_prepare(int n_tensors, float *const *params, float *const *momentum,
-                                            const void *const *grads, const int64_t *sizes, int W,
-                                            star_dtype_t grad_dtype, void *d_workspace,
-                                            size_t workspace_bytes, void *cuda_stream,
-                                            star_multi_plan_t *plan_out)
+star_status_t multi_prepare(int n_tensors, float *const *params, float *const *momentum,
+                            const void *const *grads, const int64_t *sizes, int W, star_dtype_t grad_dtype,
+                            int n_sets, void *const *snapshots, star_dtype_t snapshot_dtype,
+                            void *d_workspace, size_t workspace_bytes, void *cuda_stream,
+                            star_multi_plan_t *plan_out)
 {
     if (!plan_out) return STAR_ERR_NULL_POINTER;
     std::memset(plan_out, 0, sizeof *plan_out);
-    if (n_tensors < 0 || W < 0) return STAR_ERR_INVALID_ARG;
+    if (n_tensors < 0 || W < 0 || n_sets < 0) return STAR_ERR_INVALID_ARG;
     if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
-    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    if (snapshot_dtype != STAR_DTYPE_F32 && snapshot_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS || n_sets > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
     if (n_tensors > 0 && (!params || !momentum || !grads || !sizes)) return STAR_ERR_NULL_POINTER;
+    if (n_tensors > 0 && n_sets > 0 && !snapshots) return STAR_ERR_NULL_POINTER;
     if (!d_workspace) return STAR_ERR_NULL_POINTER;
     if (!aligned(d_workspace, kWorkspaceAlign)) return STAR_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    star_status_t st = refuse_capture(stream);
+    if (st != STAR_OK) return st;
 
     const int64_t tile = tile_elements(grad_dtype);
-    int64_t n_tiles = 0, total = 0, sizing_tiles = 0, unused = 0;
-    star_status_t st = count_tiles(n_tensors, sizes, tile, &n_tiles, &total);
+    const int full_vec = grad_dtype == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32;
+    int64_t sizing_tiles = 0, total = 0;
+    st = count_tiles(n_tensors, sizes, kTileForSizing, &sizing_tiles, &total);
     if (st != STAR_OK) return st;
-    count_tiles(n_tensors, sizes, kTileForSizing, &sizing_tiles, &unused);
-    const WorkspaceLayout need = layout_for(n_tensors, W, sizing_tiles);
-    if (workspace_bytes < need.total) return STAR_ERR_WORKSPACE_TOO_SMALL;
-    const WorkspaceLayout l = layout_for(n_tensors, W, n_tiles);
+    const WorkspaceLayout l = layout_for(n_tensors, W, n_sets, sizing_tiles);
+    if (workspace_bytes < l.total) return STAR_ERR_WORKSPACE_TOO_SMALL;
 
-    const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const unsigned gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const unsigned snap_elem = snapshot_dtype == STAR_DTYPE_BF16 ? 2 : 4;
     uint64_t complete = W == 64 ? ~uint64_t{0} : ((uint64_t{1} << W) - 1);
     std::vector<unsigned char> host(l.total, 0);
+    std::vector<Interval> intervals;
+    intervals.reserve(static_cast<size_t>(n_tensors) * static_cast<size_t>(2 + W + n_sets));
     TensorEntry *entries = reinterpret_cast<TensorEntry *>(host.data() + l.tensors_off);
     const void **table = reinterpret_cast<const void **>(host.data() + l.grads_off);
+    void **snap_table = reinterpret_cast<void **>(host.data() + l.snaps_off);
     int32_t *tile_tensor = reinterpret_cast<int32_t *>(host.data() + l.tiles_off);
     int64_t next_tile = 0;
     for (int t = 0; t < n_tensors; ++t) {
@@ -459,15 +589,17 @@ extern "C" star_status_t star_multi_prepare(int n_tensors, float *const *params,
         e.momentum = momentum[t];
         e.size = size;
         e.first_tile = next_tile;
-        e.pad = 0;
-        Alignment align;
+        Buffers buffers;
+        auto note = [&](const void *ptr, unsigned elem, bool written) {
+            const uintptr_t a = reinterpret_cast<uintptr_t>(ptr);
+            intervals.push_back(Interval{a, a + static_cast<uintptr_t>(size) * elem, written});
+            buffers.add(ptr, elem);
+        };
         if (size > 0) {
             if (!params[t] || !momentum[t]) return STAR_ERR_NULL_POINTER;
             if (!aligned(params[t], 4) || !aligned(momentum[t], 4)) return STAR_ERR_INVALID_ARG;
-            const size_t state_bytes = static_cast<size_t>(size) * 4;
-            if (overlaps(params[t], state_bytes, momentum[t], state_bytes)) return STAR_ERR_INVALID_ARG;
-            align.add_state(params[t]);
-            align.add_state(momentum[t]);
+            note(params[t], 4, true);
+            note(momentum[t], 4, true);
         }
         for (int w = 0; w < W; ++w) {
             const void *g = grads[static_cast<size_t>(t) * W + w];
@@ -478,76 +610,161 @@ extern "C" star_status_t star_multi_prepare(int n_tensors, float *const *params,
                 continue;
             }
             if (!aligned(g, gsize)) return STAR_ERR_INVALID_ARG;
-            const size_t state_bytes = static_cast<size_t>(size) * 4, grad_bytes = static_cast<size_t>(size) * gsize;
-            if (overlaps(g, grad_bytes, params[t], state_bytes) || overlaps(g, grad_bytes, momentum[t], state_bytes))
-                return STAR_ERR_INVALID_ARG;
-            align.add_grad(g);
+            note(g, gsize, false);
         }
-        e.vec = vector_width(grad_dtype, align);
-        const int64_t tiles_here = (size + tile - 1) / tile;
+        for (int set = 0; set < n_sets; ++set) {
+            void *snap = snapshots[static_cast<size_t>(t) * n_sets + set];
+            snap_table[static_cast<size_t>(t) * n_sets + set] = snap;
+            if (size == 0 || !snap) continue;
+            if (!aligned(snap, snap_elem)) return STAR_ERR_INVALID_ARG;
+            note(snap, snap_elem, true);
+        }
+        const VectorPlan plan = plan_vector(grad_dtype, buffers, size, false);
+        e.vec = plan.vec == full_vec ? full_vec : 1;
+        e.head = e.vec == full_vec ? plan.head : 0;
+        const int64_t tiles_here = (size - e.head + tile - 1) / tile + (e.head > 0 ? 1 : 0);
         for (int64_t i = 0; i < tiles_here; ++i) tile_tensor[next_tile + i] = t;
         next_tile += tiles_here;
     }
+    if (!written_buffers_are_disjoint(intervals)) return STAR_ERR_INVALID_ARG;
 
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const cudaError_t e = cudaMemcpyAsync(d_workspace, host.data(), l.total, cudaMemcpyHostToDevice, stream);
+    const size_t used = round_up(l.tiles_off + sizeof(int32_t) * static_cast<size_t>(next_tile), kWorkspaceAlign);
+    const cudaError_t e = cudaMemcpyAsync(d_workspace, host.data(), std::min(used, l.total), cudaMemcpyHostToDevice,
+                                          stream);
     if (e != cudaSuccess) return cuda_failed(e);
 
     plan_out->magic = kPlanMagic;
     plan_out->d_workspace = d_workspace;
     plan_out->total_elements = total;
-    plan_out->n_tiles = n_tiles;
+    plan_out->n_tiles = next_tile;
     plan_out->complete_workers = complete;
     plan_out->n_tensors = n_tensors;
     plan_out->W = W;
     plan_out->grad_dtype = static_cast<int32_t>(grad_dtype);
     plan_out->tile_elements = static_cast<int32_t>(tile);
+    plan_out->n_snapshot_sets = n_sets;
+    plan_out->snapshot_dtype = static_cast<int32_t>(snapshot_dtype);
     return STAR_OK;
 }
 
-namespace {
-
-star_status_t update_multi(const star_multi_plan_t *plan, const int32_t *group_offsets,
-                           const int32_t *group_members, int n_groups, float lr, const float *lrs, float mu,
-                           float wd, void *cuda_stream);
-
 }  // namespace
 
-extern "C" star_status_t star_group_update_multi(const star_multi_plan_t *plan,
-                                                 const int32_t *group_offsets, const int32_t *group_members,
-                                                 int n_groups, float lr, float mu, float wd,
-                                                 void *cuda_stream)
+extern "C" star_status_t star_multi_workspace_bytes_ex(int n_tensors, const int64_t *sizes, int W,
+                                                       int n_snapshot_sets, size_t *bytes_out)
 {
-    return update_multi(plan, group_offsets, group_members, n_groups, lr, nullptr, mu, wd, cuda_stream);
+    if (!bytes_out) return STAR_ERR_NULL_POINTER;
+    if (n_tensors < 0 || W < 0 || n_snapshot_sets < 0) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS || n_snapshot_sets > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    if (n_tensors > 0 && !sizes) return STAR_ERR_NULL_POINTER;
+    int64_t n_tiles = 0, total = 0;
+    const star_status_t st = count_tiles(n_tensors, sizes, kTileForSizing, &n_tiles, &total);
+    if (st != STAR_OK) return st;
+    *bytes_out = layout_for(n_tensors, W, n_snapshot_sets, n_tiles).total;
+    return STAR_OK;
 }
 
-extern "C" star_status_t star_group_update_multi_lrs(const star_multi_plan_t *plan,
-                                                     const int32_t *group_offsets,
-                                                     const int32_t *group_members, int n_groups,
-                                                     const float *lrs, float mu, float wd, void *cuda_stream)
+extern "C" star_status_t star_multi_workspace_bytes(int n_tensors, const int64_t *sizes, int W,
+                                                    size_t *bytes_out)
 {
-    if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
-    return update_multi(plan, group_offsets, group_members, n_groups, 0.0f, lrs, mu, wd, cuda_stream);
+    return star_multi_workspace_bytes_ex(n_tensors, sizes, W, 0, bytes_out);
+}
+
+extern "C" star_status_t star_multi_prepare(int n_tensors, float *const *params, float *const *momentum,
+                                            const void *const *grads, const int64_t *sizes, int W,
+                                            star_dtype_t grad_dtype, void *d_workspace,
+                                            size_t workspace_bytes, void *cuda_stream,
+                                            star_multi_plan_t *plan_out)
+{
+    return multi_prepare(n_tensors, params, momentum, grads, sizes, W, grad_dtype, 0, nullptr, STAR_DTYPE_F32,
+                         d_workspace, workspace_bytes, cuda_stream, plan_out);
+}
+
+extern "C" star_status_t star_multi_prepare_ex(int n_tensors, float *const *params, float *const *momentum,
+                                               const void *const *grads, const int64_t *sizes, int W,
+                                               star_dtype_t grad_dtype, int n_snapshot_sets,
+                                               void *const *snapshots, star_dtype_t snapshot_dtype,
+                                               void *d_workspace, size_t workspace_bytes, void *cuda_stream,
+                                               star_multi_plan_t *plan_out)
+{
+    return multi_prepare(n_tensors, params, momentum, grads, sizes, W, grad_dtype, n_snapshot_sets, snapshots,
+                         snapshot_dtype, d_workspace, workspace_bytes, cuda_stream, plan_out);
 }
 
 namespace {
 
+template <typename Kernel, typename Args>
+star_status_t launch_tiles(Kernel kernel, Geometry *cache, const Args &args, int64_t n_tiles, cudaStream_t stream)
+{
+    int blocks = 0;
+    cudaError_t e = resident_blocks(kernel, cache, &blocks);
+    if (e != cudaSuccess) return cuda_failed(e);
+    // The tile-map kernel pays a table lookup per block: measured on B200 the
+    // persistent grid is the faster shape for it at every list size tried.
+    const int grid = static_cast<int>(n_tiles < blocks ? n_tiles : blocks);
+    kernel<<<grid, kBlockThreads, 0, stream>>>(args);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_failed(e);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return STAR_OK;
+}
+
+template <typename G, int VEC>
+star_status_t launch_multi(const MultiArgs &args, cudaStream_t stream)
+{
+    static Geometry cache[kMaxDevices];
+    return launch_tiles(star_update_multi_kernel<G, VEC, kDepthVector>, cache, args, args.n_tiles, stream);
+}
+
+template <typename G, int VEC, int TREE>
+star_status_t launch_multi_ex(const MultiExArgs &args, cudaStream_t stream)
+{
+    static Geometry cache[kMaxDevices];
+    return launch_tiles(star_update_multi_ex_kernel<G, VEC, kDepthVector, TREE>, cache, args, args.base.n_tiles,
+                        stream);
+}
+
+template <typename G, int VEC>
+star_status_t dispatch_multi_ex(const MultiExArgs &args, int tree, cudaStream_t stream)
+{
+    switch (tree) {
+    case 4: return launch_multi_ex<G, VEC, 4>(args, stream);
+    case 16: return launch_multi_ex<G, VEC, 16>(args, stream);
+    case 64: return launch_multi_ex<G, VEC, 64>(args, stream);
+    default: return launch_multi_ex<G, VEC, 0>(args, stream);
+    }
+}
+
+// One round over a prepared list.  snapshot_set_of_group == nullptr and the
+// linear order take the plain kernel.
 star_status_t update_multi(const star_multi_plan_t *plan, const int32_t *group_offsets,
                            const int32_t *group_members, int n_groups, float lr, const float *lrs, float mu,
-                           float wd, void *cuda_stream)
+                           float wd, const int32_t *snapshot_set_of_group, star_sum_order_t sum_order,
+                           void *cuda_stream)
 {
     if (!plan) return STAR_ERR_NULL_POINTER;
     if (plan->magic != kPlanMagic || !plan->d_workspace) return STAR_ERR_INVALID_ARG;
-    MultiArgs args;
+    if (sum_order != STAR_SUM_LINEAR && sum_order != STAR_SUM_TREE) return STAR_ERR_INVALID_ARG;
+    MultiExArgs ex;
+    MultiArgs &args = ex.base;
     const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, plan->W, lr, &args.sched, lrs);
     if (st != STAR_OK) return st;
+    bool any_snapshot = false;
+    std::memset(ex.snapshot_set, -1, sizeof ex.snapshot_set);
+    for (int k = 0; snapshot_set_of_group && k < n_groups; ++k) {
+        const int set = snapshot_set_of_group[k];
+        if (set < -1 || set >= plan->n_snapshot_sets) return STAR_ERR_INVALID_ARG;
+        if (set < 0) continue;
+        ex.snapshot_set[group_offsets[k + 1] - 1] = static_cast<int8_t>(set);
+        any_snapshot = true;
+    }
     if (plan->n_tiles == 0 || n_groups == 0) return STAR_OK;
     for (int j = 0; j < args.sched.n_slots; ++j)
         if (!(plan->complete_workers >> args.sched.member[j] & 1u)) return STAR_ERR_NULL_POINTER;
 
     const star_dtype_t dt = static_cast<star_dtype_t>(plan->grad_dtype);
-    const int64_t sizing_tiles = plan->n_tiles;     // layout offsets depend on n_tensors and W only up to tiles_off
-    const WorkspaceLayout l = layout_for(plan->n_tensors, plan->W, sizing_tiles);
+    if (dt != STAR_DTYPE_BF16 && dt != STAR_DTYPE_F32) return STAR_ERR_INVALID_ARG;
+    // the offsets of the tables do not depend on the number of tiles
+    const WorkspaceLayout l = layout_for(plan->n_tensors, plan->W, plan->n_snapshot_sets, plan->n_tiles);
     const char *base = static_cast<const char *>(plan->d_workspace);
     args.tensors = reinterpret_cast<const TensorEntry *>(base + l.tensors_off);
     args.grads = reinterpret_cast<const void *const *>(base + l.grads_off);
@@ -556,12 +773,49 @@ star_status_t update_multi(const star_multi_plan_t *plan, const int32_t *group_o
     args.W = plan->W;
     args.hyper = Hyper{mu, wd};
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (dt == STAR_DTYPE_BF16) return launch_multi<GradBF16, kVecBF16>(args, stream);
-    if (dt == STAR_DTYPE_F32) return launch_multi<GradF32, kVecF32>(args, stream);
-    return STAR_ERR_INVALID_ARG;
+    const int tree = tree_span(sum_order, largest_group(group_offsets, n_groups));
+    if (tree == 0 && !any_snapshot)
+        return dt == STAR_DTYPE_BF16 ? launch_multi<GradBF16, kVecBF16>(args, stream)
+                                     : launch_multi<GradF32, kVecF32>(args, stream);
+    ex.snapshots = reinterpret_cast<void *const *>(base + l.snaps_off);
+    ex.n_sets = plan->n_snapshot_sets;
+    ex.snapshot_bf16 = plan->snapshot_dtype == STAR_DTYPE_BF16 ? 1 : 0;
+    return dt == STAR_DTYPE_BF16 ? dispatch_multi_ex<GradBF16, kVecBF16>(ex, tree, stream)
+                                 : dispatch_multi_ex<GradF32, kVecF32>(ex, tree, stream);
 }
 
 }  // namespace
+
+extern "C" star_status_t star_group_update_multi(const star_multi_plan_t *plan,
+                                                 const int32_t *group_offsets, const int32_t *group_members,
+                                                 int n_groups, float lr, float mu, float wd,
+                                                 void *cuda_stream)
+{
+    return update_multi(plan, group_offsets, group_members, n_groups, lr, nullptr, mu, wd, nullptr, STAR_SUM_LINEAR,
+                        cuda_stream);
+}
+
+extern "C" star_status_t star_group_update_multi_lrs(const star_multi_plan_t *plan,
+                                                     const int32_t *group_offsets,
+                                                     const int32_t *group_members, int n_groups,
+                                                     const float *lrs, float mu, float wd, void *cuda_stream)
+{
+    if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
+    return update_multi(plan, group_offsets, group_members, n_groups, 0.0f, lrs, mu, wd, nullptr, STAR_SUM_LINEAR,
+                        cuda_stream);
+}
+
+extern "C" star_status_t star_group_update_multi_ex(const star_multi_plan_t *plan,
+                                                    const int32_t *group_offsets,
+                                                    const int32_t *group_members, int n_groups,
+                                                    const float *lrs, float mu, float wd,
+                                                    const int32_t *snapshot_set_of_group,
+                                                    star_sum_order_t sum_order, void *cuda_stream)
+{
+    if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
+    return update_multi(plan, group_offsets, group_members, n_groups, 0.0f, lrs, mu, wd, snapshot_set_of_group,
+                        sum_order, cuda_stream);
+}
 
 // ---------------------------------------------------------------------------
 // Host-resident state and gradients: chunked, double-buffered streaming.
@@ -709,7 +963,9 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
         args.params = d_p;
         args.momentum = d_v;
         args.n = count;
-        const star_status_t ls = dispatch_flat(args, grad_dtype, Alignment{}, stream);   // staging buffers are aligned
+        // staging buffers are aligned: full vector width, no leading elements
+        const star_status_t ls = dispatch_flat(
+            args, grad_dtype, VectorPlan{grad_dtype == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32, 0}, stream);
         if (ls != STAR_OK) return ls;
         e = cudaEventRecord(hp->kernel_done[b], stream);
         if (e != cudaSuccess) return cuda_failed(e);
@@ -768,8 +1024,12 @@ extern "C" star_status_t star_group_update_multi_noalloc(
     const int64_t *sizes, int W, star_dtype_t grad_dtype, const int32_t *group_offsets,
     const int32_t *group_members, int n_groups, float lr, float mu, float wd, void *cuda_stream)
 {
+    // Inside a stream capture nothing is enqueued (the table copy reads host
+    // memory that is gone by the time a graph would replay it).
+    star_status_t st = refuse_capture(static_cast<cudaStream_t>(cuda_stream));
+    if (st != STAR_OK) return st;
     // Reject a bad schedule before the shared table is touched.
-    star_status_t st = star_schedule_validate(group_offsets, group_members, n_groups, W);
+    st = star_schedule_validate(group_offsets, group_members, n_groups, W);
     if (st != STAR_OK) return st;
     size_t need = 0;
     st = star_multi_workspace_bytes(n_tensors, sizes, W, &need);

@@ -28,13 +28,16 @@ constexpr int kBlockThreads = 256;
 constexpr int kResidentBlocks = 4;
 
 // The schedule as the kernel sees it: one slot per scheduled worker, in the
-// order the gradients are consumed.  A slot that closes a group carries that
-// group's size and (negated) learning rate.
+// order the gradients are consumed.  A slot that closes a group carries the
+// divisor of that group's mean (the group's size; for an update from partial
+// sums, the number of gradient reports behind them) and its (negated)
+// learning rate; the slot that opens a group carries the group's size for the
+// kernels that walk the schedule group by group (tree order).
 struct FlatSchedule {
     int32_t n_slots;
     uint8_t member[kMaxWorkers];       // slot -> worker index
-    uint8_t group_size[kMaxWorkers];   // |G_k| on the last slot of group k, else 0
-    uint8_t index_in_group[kMaxWorkers];   // position of the slot inside its group (tree order only)
+    uint8_t group_size[kMaxWorkers];   // divisor of the mean on the last slot of group k, else 0
+    uint8_t size_at_start[kMaxWorkers];    // |G_k| on the first slot of group k, else 0
     float neg_lr[kMaxWorkers];         // -lr_k on the last slot of group k
 };
 
@@ -190,46 +193,133 @@ __device__ __forceinline__ void apply_update(float (&p)[VEC], float (&v)[VEC], c
     }
 }
 
+// after_group(slot, first, p) is called right after the update of the group that
+// closes on `slot`, with the parameters as they stand then.
+struct NoSnapshot {
+    template <int VEC> __device__ __forceinline__ void operator()(int, int64_t, const float (&)[VEC]) const {}
+};
+
+template <int VEC> __device__ __forceinline__ void add_rows(float (&a)[VEC], const float (&b)[VEC])
+{
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) a[e] = __fadd_rn(a[e], b[e]);
+}
+
+// ---------------------------------------------------------------------------
+// Pairwise (tree) summation order, as gradients are combined along a binary
+// aggregation tree (Section IV-D2b): tree(m_0..m_{c-1}) is the member itself
+// for c = 1, else tree(first h) + tree(remaining c - h) with h the largest
+// power of two below c.  Over an aligned span of N = 2^k slots of which the
+// first `count` are used that is
+//     count <= N/2 : the tree over the first half
+//     else         : (full tree over the first half) + (tree over the count - N/2
+//                    used slots of the second half)
+// so a group is summed by halving with no per-leaf bookkeeping.  Spans of up to
+// BLOCK slots are a leaf block: its gradient loads are issued back to back and
+// added straight from their registers; each level above a block keeps one
+// partial sum (a row of VEC registers).
+// ---------------------------------------------------------------------------
+
+// Leaves LO .. LO + N - 1 of a loaded block, of which the first r (1..N) are used.
+template <typename G, int VEC, int LO, int N, int BLOCK>
+__device__ __forceinline__ void leaf_tree(const Raw<VEC * G::kBytes> (&raw)[BLOCK], int r, float (&out)[VEC])
+{
+    if constexpr (N == 1) {
+        G::template widen<VEC>(raw[LO], out);
+    } else {
+        constexpr int H = N / 2;
+        leaf_tree<G, VEC, LO, H, BLOCK>(raw, min(r, H), out);
+        if (r > H) {
+            float t[VEC];
+            leaf_tree<G, VEC, LO + H, H, BLOCK>(raw, r - H, t);
+            add_rows<VEC>(out, t);
+        }
+    }
+}
+
+// Tree-order sum of slots base .. base + count - 1, 1 <= count <= N.
+template <typename G, int VEC, int N, int BLOCK, typename GradPtr>
+__device__ __forceinline__ void tree_sum(GradPtr grad_ptr, int64_t first, int base, int count, float (&out)[VEC])
+{
+    if constexpr (N <= BLOCK) {
+        constexpr int GB = VEC * G::kBytes;
+        Raw<GB> raw[N];
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            if (j < count) {
+                const char *g = static_cast<const char *>(grad_ptr(base + j));
+                raw[j] = load_stream<GB>(g + first * G::kBytes);
+            }
+        }
+        leaf_tree<G, VEC, 0, N, N>(raw, count, out);
+    } else {
+        constexpr int H = N / 2;
+        tree_sum<G, VEC, H, BLOCK>(grad_ptr, first, base, min(count, H), out);
+        if (count > H) {
+            float t[VEC];
+            tree_sum<G, VEC, H, BLOCK>(grad_ptr, first, base + H, count - H, t);
+            add_rows<VEC>(out, t);
+        }
+    }
+}
+
+// Leaf block of the tree kernels: the kernel for groups of up to 4 members
+// loads a whole group at once and runs at the occupancy of the linear kernels;
+// the kernels for larger groups load 8 gradients at a time and run two blocks
+// per SM (the rows of partial sums cost registers; the deeper loads keep as
+// many bytes in flight per SM).
+__host__ __device__ constexpr int tree_block(int tree) { return tree <= 4 ? 4 : 8; }
+
+// Tree-order sum of one group of c <= TREE members whose first slot is `start`.
+// Up to two leaf blocks the halving is written out; beyond (groups of up to 64
+// members: up to 8 blocks of 8) the blocks are walked by a loop that keeps the
+// partial sums of the levels above a block as a binary counter -- after b
+// blocks the set bits of b are the pending levels; a new block merges with the
+// pending levels below its first clear bit, the last block with every pending
+// level in ascending order -- which is the same tree.  (Writing all eight
+// blocks out made the compiler hold every gradient pointer in registers.)
+template <typename G, int VEC, int TREE, typename GradPtr>
+__device__ __forceinline__ void group_tree_sum(GradPtr grad_ptr, int64_t first, int start, int c, float (&out)[VEC])
+{
+    constexpr int BLOCK = tree_block(TREE);
+    if constexpr (TREE <= 2 * BLOCK) {
+        tree_sum<G, VEC, TREE, BLOCK>(grad_ptr, first, start, c, out);
+    } else {
+        static_assert(TREE == 8 * BLOCK, "the block loop keeps three pending levels");
+        float pend0[VEC], pend1[VEC], pend2[VEC];
+#pragma unroll 1
+        for (int b = 0; b * BLOCK < c; ++b) {
+            const int left = c - b * BLOCK;
+            tree_sum<G, VEC, BLOCK, BLOCK>(grad_ptr, first, start + b * BLOCK, min(left, BLOCK), out);
+            if (left > BLOCK) {                      // not the last block: b <= 6
+                if ((b & 1) == 0) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) pend0[e] = out[e];
+                } else if ((b & 2) == 0) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) pend1[e] = __fadd_rn(pend0[e], out[e]);
+                } else {                             // b == 3: levels 0 and 1 are pending
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) pend2[e] = __fadd_rn(pend1[e], __fadd_rn(pend0[e], out[e]));
+                }
+            } else {
+                if (b & 1) add_rows<VEC>(out, pend0);
+                if (b & 2) add_rows<VEC>(out, pend1);
+                if (b & 4) add_rows<VEC>(out, pend2);
+            }
+        }
+    }
+}
+
 // All groups of the round on the VEC elements starting at element `first` of
 // one tensor.  grad_ptr(slot) returns the base pointer of the slot's worker;
 // state_ptr(0) / state_ptr(1) return the tensor's params / momentum base and are
 // asked again at store time, so that a caller whose bases live in memory need
 // not hold them in registers across the update.
 //
-// after_group(slot, p) is called right after the update of the group that
-// closes on `slot`, with the parameters as they stand then.
-struct NoSnapshot {
-    template <int VEC> __device__ __forceinline__ void operator()(int, int64_t, const float (&)[VEC]) const {}
-};
-
-//
-// TREE selects the in-group summation order.  false: left to right.  true:
-// pairwise, as along a binary aggregation tree (Section IV-D2b): the partial
-// sums pending after i leaves are the set bits of i (level l spans 2^l
-// leaves); a new leaf merges with the pending levels below its first clear
-// bit, the group's last leaf with every pending level in ascending order.
-// That is tree(first h) + tree(rest) with h the largest power of two below the
-// group size.  A group of c members needs ceil(log2(c)) pending levels of VEC
-// registers each, so the tree kernels are instantiated for 2, 4 and 6 levels
-// (groups of up to 4, 16 and 64 members) and compiled for 3, 3 and 2 resident
-// blocks; TREE is the number of levels, 0 = linear order.
-
-// Merge a new leaf with the pending partial sums of levels 0..LEVEL-1 and park
-// the result on LEVEL.
-template <int LEVEL, int VEC, int ROWS>
-__device__ __forceinline__ void tree_merge(float (&pending)[ROWS][VEC], float (&f)[VEC])
-{
-    if constexpr (LEVEL < ROWS) {
-#pragma unroll
-        for (int l = 0; l < LEVEL; ++l) {
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) f[e] = __fadd_rn(pending[l][e], f[e]);
-        }
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) pending[LEVEL][e] = f[e];
-    }
-}
-
+// TREE = 0: in-group sums run left to right; the flattened schedule is walked
+// in chunks of DEPTH slots whatever group they belong to.  TREE = 4, 16 or 64:
+// tree order for groups of up to TREE members, walked group by group.
 template <typename G, int VEC, int DEPTH, int TREE = 0, typename StatePtr, typename GradPtr,
           typename AfterGroup = NoSnapshot>
 __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first, const FlatSchedule &s,
@@ -237,82 +327,62 @@ __device__ __forceinline__ void update_vector(StatePtr state_ptr, int64_t first,
                                               AfterGroup after_group = AfterGroup())
 {
     constexpr int GB = VEC * G::kBytes;
-    float p[VEC], v[VEC], sum[VEC];
-    constexpr int kTreeLevels = TREE;
-    [[maybe_unused]] float pending[TREE > 0 ? TREE : 1][VEC];
+    float p[VEC], v[VEC];
     load_state<VEC>(state_ptr(0) + first, p);
     load_state<VEC>(state_ptr(1) + first, v);
-    // -0.0f is the additive identity of IEEE addition (x + -0 == x for every x,
-    // including x == -0), so a running sum started there equals the plain
-    // left-to-right sum that starts at the first member.
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) sum[e] = -0.0f;
-
     const int n_slots = s.n_slots;
-    for (int base = 0; base < n_slots; base += DEPTH) {
-        Raw<GB> raw[DEPTH];
+
+    if constexpr (TREE > 0) {
+        for (int start = 0; start < n_slots;) {
+            const int c = max(static_cast<int>(s.size_at_start[start]), 1);
+            const int closing = start + c - 1;
+            float sum[VEC];
+            group_tree_sum<G, VEC, TREE>(grad_ptr, first, start, c, sum);
+            if (c > 1) {
+                const float count = static_cast<float>(s.group_size[closing]);
 #pragma unroll
-        for (int j = 0; j < DEPTH; ++j) {
-            if (base + j < n_slots) {
-                const char *g = static_cast<const char *>(grad_ptr(base + j));
-                raw[j] = load_stream<GB>(g + first * G::kBytes);
+                for (int e = 0; e < VEC; ++e) sum[e] = exact_mean(sum[e], count);
             }
+            apply_update<VEC>(p, v, sum, s.neg_lr[closing], h);
+            after_group.template operator()<VEC>(closing, first, p);
+            start += c;
         }
+    } else {
+        // -0.0f is the additive identity of IEEE addition (x + -0 == x for every x,
+        // including x == -0), so a running sum started there equals the plain
+        // left-to-right sum that starts at the first member.
+        float sum[VEC];
 #pragma unroll
-        for (int j = 0; j < DEPTH; ++j) {
-            if (base + j < n_slots) {
-                float f[VEC];
-                G::template widen<VEC>(raw[j], f);
-                const int gs = s.group_size[base + j];
-                if (gs == 1) {                       // singleton group: the mean is the gradient
-                    apply_update<VEC>(p, v, f, s.neg_lr[base + j], h);
-                    after_group.template operator()<VEC>(base + j, first, p);
-                } else if constexpr (TREE > 0) {
-                    const int leaves_before = s.index_in_group[base + j];
-                    if (gs == 0) {                   // not the last leaf: merge up to the first clear bit
-                        // A real (warp-uniform) branch per level, most frequent level
-                        // first: predicating all levels on every leaf made this path
-                        // issue-bound, and a jump table was slower than this chain.
-                        const int level = __ffs(~leaves_before) - 1;      // number of trailing set bits
-                        if (level == 0) {
-                            tree_merge<0, VEC>(pending, f);
-                        } else if (level == 1) {
-                            tree_merge<1, VEC>(pending, f);
-                        } else if constexpr (TREE > 2) {
-                            if (level == 2) {
-                                tree_merge<2, VEC>(pending, f);
-                            } else if (level == 3) {
-                                tree_merge<3, VEC>(pending, f);
-                            } else if constexpr (TREE > 4) {
-                                if (level == 4) tree_merge<4, VEC>(pending, f);
-                                else tree_merge<5, VEC>(pending, f);
-                            }
-                        }
-                    } else {                         // last leaf: fold every pending level
+        for (int e = 0; e < VEC; ++e) sum[e] = -0.0f;
+        for (int base = 0; base < n_slots; base += DEPTH) {
+            Raw<GB> raw[DEPTH];
 #pragma unroll
-                        for (int l = 0; l < kTreeLevels; ++l) {
-                            if (leaves_before >> l & 1) {
+            for (int j = 0; j < DEPTH; ++j) {
+                if (base + j < n_slots) {
+                    const char *g = static_cast<const char *>(grad_ptr(base + j));
+                    raw[j] = load_stream<GB>(g + first * G::kBytes);
+                }
+            }
 #pragma unroll
-                                for (int e = 0; e < VEC; ++e) f[e] = __fadd_rn(pending[l][e], f[e]);
-                            }
-                        }
-                        const float count = static_cast<float>(gs);
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e) f[e] = exact_mean(f[e], count);
+            for (int j = 0; j < DEPTH; ++j) {
+                if (base + j < n_slots) {
+                    float f[VEC];
+                    G::template widen<VEC>(raw[j], f);
+                    const int gs = s.group_size[base + j];
+                    if (gs == 1) {                       // singleton group: the mean is the gradient
                         apply_update<VEC>(p, v, f, s.neg_lr[base + j], h);
                         after_group.template operator()<VEC>(base + j, first, p);
-                    }
-                } else {
+                    } else {
+                        add_rows<VEC>(sum, f);
+                        if (gs != 0) {
+                            const float count = static_cast<float>(gs);
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) sum[e] = __fadd_rn(sum[e], f[e]);
-                    if (gs != 0) {
-                        const float count = static_cast<float>(gs);
+                            for (int e = 0; e < VEC; ++e) sum[e] = exact_mean(sum[e], count);
+                            apply_update<VEC>(p, v, sum, s.neg_lr[base + j], h);
+                            after_group.template operator()<VEC>(base + j, first, p);
 #pragma unroll
-                        for (int e = 0; e < VEC; ++e) sum[e] = exact_mean(sum[e], count);
-                        apply_update<VEC>(p, v, sum, s.neg_lr[base + j], h);
-                        after_group.template operator()<VEC>(base + j, first, p);
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e) sum[e] = -0.0f;
+                            for (int e = 0; e < VEC; ++e) sum[e] = -0.0f;
+                        }
                     }
                 }
             }
@@ -330,27 +400,41 @@ struct FlatArgs {
     float *momentum;
     const void *grads[kMaxWorkers];
     int64_t n;
+    int32_t head;          // leading elements (< VEC) done one by one; the vector body starts there
     FlatSchedule sched;
     Hyper hyper;
 };
 
-// Vector kernel: requires 32-byte aligned bases (p and v move in 32-byte accesses when VEC = 8).
-// Grid-stride over vectors; the last < VEC elements are done one by one by the
-// first threads of block 0.
+// The elements of a flat tensor that the vector body [head, head + n_vec * VEC)
+// leaves over -- up to VEC - 1 in front of it (buffers that are views at an odd
+// element offset into aligned storage reach vector alignment only there) and
+// up to VEC - 1 behind it -- are done one by one by the first 2 * VEC threads
+// of block 0.  Returns the element this thread owns, or -1.
+template <int VEC>
+__device__ __forceinline__ int64_t edge_element(int64_t n, int head, int64_t n_vec)
+{
+    if (blockIdx.x != 0 || threadIdx.x >= 2 * VEC) return -1;
+    const int t = threadIdx.x;
+    if (t < VEC) return t < head ? t : -1;
+    const int64_t e = head + n_vec * VEC + (t - VEC);
+    return e < n ? e : -1;
+}
+
+// Vector kernel: requires bases that are vector-aligned at element `head`
+// (32 bytes for p and v when VEC = 8).  Grid-stride over vectors.
 template <typename G, int VEC, int DEPTH>
 __global__ void __launch_bounds__(kBlockThreads, kResidentBlocks)
 star_update_flat_kernel(const __grid_constant__ FlatArgs a)
 {
-    const int64_t n_vec = a.n / VEC;
+    const int64_t n_vec = (a.n - a.head) / VEC;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlockThreads;
     auto grad_ptr = [&](int slot) -> const void * { return a.grads[a.sched.member[slot]]; };
     auto state_ptr = [&](int which) -> float * { return which == 0 ? a.params : a.momentum; };
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kBlockThreads + threadIdx.x; i < n_vec; i += stride)
-        update_vector<G, VEC, DEPTH>(state_ptr, i * VEC, a.sched, a.hyper, grad_ptr);
+        update_vector<G, VEC, DEPTH>(state_ptr, a.head + i * VEC, a.sched, a.hyper, grad_ptr);
     if constexpr (VEC > 1) {
-        const int64_t tail = n_vec * VEC + threadIdx.x;
-        if (blockIdx.x == 0 && threadIdx.x < VEC && tail < a.n)
-            update_vector<G, 1, DEPTH>(state_ptr, tail, a.sched, a.hyper, grad_ptr);
+        const int64_t e = edge_element<VEC>(a.n, a.head, n_vec);
+        if (e >= 0) update_vector<G, 1, DEPTH>(state_ptr, e, a.sched, a.hyper, grad_ptr);
     }
 }
 
@@ -404,9 +488,11 @@ struct StoreSnapshot {
     }
 };
 
-constexpr int tree_resident_blocks(int levels)
+// Resident blocks the extended kernels are compiled for: the tree order keeps
+// one more row of partial sums per level of four.
+constexpr int tree_resident_blocks(int tree)
 {
-    return levels == 0 ? kResidentBlocks : levels <= 4 ? 3 : 2;
+    return tree <= 4 ? kResidentBlocks : 2;
 }
 
 template <typename G, int VEC, int DEPTH, int TREE>
@@ -414,33 +500,95 @@ __global__ void __launch_bounds__(kBlockThreads, tree_resident_blocks(TREE))
 star_update_flat_snapshot_kernel(const __grid_constant__ SnapshotArgs a)
 {
     const FlatArgs &f = a.flat;
-    const int64_t n_vec = f.n / VEC;
+    const int64_t n_vec = (f.n - f.head) / VEC;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlockThreads;
     auto grad_ptr = [&](int slot) -> const void * { return f.grads[f.sched.member[slot]]; };
     auto state_ptr = [&](int which) -> float * { return which == 0 ? f.params : f.momentum; };
     const StoreSnapshot snap{&a};
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kBlockThreads + threadIdx.x; i < n_vec; i += stride)
-        update_vector<G, VEC, DEPTH, TREE>(state_ptr, i * VEC, f.sched, f.hyper, grad_ptr, snap);
+        update_vector<G, VEC, DEPTH, TREE>(state_ptr, f.head + i * VEC, f.sched, f.hyper, grad_ptr, snap);
     if constexpr (VEC > 1) {
-        const int64_t tail = n_vec * VEC + threadIdx.x;
-        if (blockIdx.x == 0 && threadIdx.x < VEC && tail < f.n)
-            update_vector<G, 1, DEPTH, TREE>(state_ptr, tail, f.sched, f.hyper, grad_ptr, snap);
+        const int64_t e = edge_element<VEC>(f.n, f.head, n_vec);
+        if (e >= 0) update_vector<G, 1, DEPTH, TREE>(state_ptr, e, f.sched, f.hyper, grad_ptr, snap);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Sum of a list of gradient buffers (all-reduce architecture, Section IV-B: a
+// parent adds its children's gradients to its own before the ring): out[i] =
+// src[0][i] + src[1][i] + ... in binary32, left to right (TREE = 0) or in tree
+// order, stored as binary32 or rounded to bf16.  Every source element is read
+// once, every output element written once.
+// ---------------------------------------------------------------------------
+struct ReduceArgs {
+    void *out;
+    const void *src[kMaxWorkers];      // in summation order
+    int64_t n;
+    int32_t count;
+    int32_t head;
+    int32_t out_bf16;
+};
+
+template <typename G, int VEC, int DEPTH, int TREE>
+__device__ __forceinline__ void reduce_vector(const ReduceArgs &a, int64_t first)
+{
+    constexpr int GB = VEC * G::kBytes;
+    float sum[VEC];
+    auto grad_ptr = [&](int slot) -> const void * { return a.src[slot]; };
+    if constexpr (TREE > 0) {
+        group_tree_sum<G, VEC, TREE>(grad_ptr, first, 0, a.count, sum);
+    } else {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) sum[e] = -0.0f;
+        for (int base = 0; base < a.count; base += DEPTH) {
+            Raw<GB> raw[DEPTH];
+#pragma unroll
+            for (int j = 0; j < DEPTH; ++j)
+                if (base + j < a.count)
+                    raw[j] = load_stream<GB>(static_cast<const char *>(a.src[base + j]) + first * G::kBytes);
+#pragma unroll
+            for (int j = 0; j < DEPTH; ++j) {
+                if (base + j < a.count) {
+                    float f[VEC];
+                    G::template widen<VEC>(raw[j], f);
+                    add_rows<VEC>(sum, f);
+                }
+            }
+        }
+    }
+    if (a.out_bf16) store_bf16<VEC>(static_cast<uint16_t *>(a.out) + first, sum);
+    else store_state<VEC>(static_cast<float *>(a.out) + first, sum);
+}
+
+template <typename G, int VEC, int DEPTH, int TREE>
+__global__ void __launch_bounds__(kBlockThreads, tree_resident_blocks(TREE))
+star_group_reduce_kernel(const __grid_constant__ ReduceArgs a)
+{
+    const int64_t n_vec = (a.n - a.head) / VEC;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlockThreads;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kBlockThreads + threadIdx.x; i < n_vec; i += stride)
+        reduce_vector<G, VEC, DEPTH, TREE>(a, a.head + i * VEC);
+    if constexpr (VEC > 1) {
+        const int64_t e = edge_element<VEC>(a.n, a.head, n_vec);
+        if (e >= 0) reduce_vector<G, 1, DEPTH, TREE>(a, e);
     }
 }
 
 // ---------------------------------------------------------------------------
 // Tensor list.  The device workspace holds, in this order (each array 256-byte
 // aligned): per-tensor TensorEntry records, the gradient pointer table
-// [n_tensors * W], and tile_tensor[n_tiles] (tile -> tensor index).  Tiles of a
-// tensor are consecutive; TensorEntry::first_tile is the tensor's first tile.
+// [n_tensors * W], the snapshot pointer table [n_tensors * n_snapshot_sets] and
+// tile_tensor[n_tiles] (tile -> tensor index).  Tiles of a tensor are
+// consecutive; TensorEntry::first_tile is the tensor's first tile.  A tensor with
+// `head` > 0 spends its first tile on those leading elements.
 // ---------------------------------------------------------------------------
 struct TensorEntry {
     float *params;
     float *momentum;
     int64_t size;          // elements
     int64_t first_tile;
-    int32_t vec;           // elements per thread the tensor's buffer alignment allows (full width or less)
-    int32_t pad;
+    int32_t vec;           // elements per thread the tensor's buffer alignment allows (full width or 1)
+    int32_t head;          // leading elements in front of the vector-aligned body (< vec)
 };
 
 struct MultiArgs {
@@ -453,28 +601,65 @@ struct MultiArgs {
     Hyper hyper;
 };
 
-// Element-by-element path for the ragged end of a tensor and for tensors whose
-// buffers are not aligned for the full vector width.  Kept out of line: it is
-// cold, and inlining it next to the vector path costs registers there.
+// Extended tensor-list round: snapshots[t * n_sets + set] receives tensor t's
+// parameters after the group that closes on a slot with snapshot_set[slot] ==
+// set (-1: no snapshot for that group).
+struct MultiExArgs {
+    MultiArgs base;
+    void *const *snapshots;         // [n_tensors * n_sets], entries may be null
+    int32_t n_sets;
+    int32_t snapshot_bf16;
+    int8_t snapshot_set[kMaxWorkers];
+};
+
+struct NoMultiSnapshot {
+    __device__ __forceinline__ NoSnapshot for_tensor(int32_t) const { return NoSnapshot(); }
+};
+
+struct StoreMultiSnapshot {
+    const MultiExArgs *a;
+    const unsigned long long *row;     // the tensor's row of the snapshot table
+    template <int VEC> __device__ __forceinline__ void operator()(int slot, int64_t first, const float (&p)[VEC]) const
+    {
+        const int set = a->snapshot_set[slot];
+        if (set < 0) return;
+        void *dst = reinterpret_cast<void *>(__ldg(row + set));
+        if (dst == nullptr) return;
+        if (a->snapshot_bf16) store_bf16<VEC>(static_cast<uint16_t *>(dst) + first, p);
+        else store_state<VEC>(static_cast<float *>(dst) + first, p);
+    }
+};
+
+struct MultiSnapshotSource {
+    const MultiExArgs *a;
+    __device__ __forceinline__ StoreMultiSnapshot for_tensor(int32_t t) const
+    {
+        return StoreMultiSnapshot{a, reinterpret_cast<const unsigned long long *>(a->snapshots) +
+                                         static_cast<int64_t>(t) * a->n_sets};
+    }
+};
+
+// Element-by-element path for the ragged ends of a tensor and for tensors whose
+// buffers do not share a vector alignment.  Kept out of line: it is cold, and
+// inlining it next to the vector path costs registers there.
 // Handles elements first, first + step, ... below end.
-template <typename G, int DEPTH>
+template <typename G, int DEPTH, int TREE, typename After>
 __device__ __noinline__ void update_elements(const TensorEntry &te, const unsigned long long *row,
                                              int64_t first, int64_t end, int64_t step,
-                                             const FlatSchedule &s, const Hyper &h)
+                                             const FlatSchedule &s, const Hyper &h, After after)
 {
     auto grad_ptr = [&](int slot) -> const void * {
         return reinterpret_cast<const void *>(__ldg(row + s.member[slot]));
     };
     auto state_ptr = [&](int which) -> float * { return which == 0 ? te.params : te.momentum; };
     for (int64_t i = first; i < end; i += step)
-        update_vector<G, 1, DEPTH>(state_ptr, i, s, h, grad_ptr);
+        update_vector<G, 1, DEPTH, TREE>(state_ptr, i, s, h, grad_ptr, after);
 }
 
 // One block per tile of kBlockThreads * VEC elements (grid-stride over tiles);
 // a thread owns one vector of its tile.
-template <typename G, int VEC, int DEPTH>
-__global__ void __launch_bounds__(kBlockThreads, kResidentBlocks)
-star_update_multi_kernel(const __grid_constant__ MultiArgs a)
+template <typename G, int VEC, int DEPTH, int TREE, typename Snapshots>
+__device__ __forceinline__ void update_tiles(const MultiArgs &a, Snapshots snapshots)
 {
     constexpr int64_t kTile = static_cast<int64_t>(kBlockThreads) * VEC;
     for (int64_t tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
@@ -482,10 +667,14 @@ star_update_multi_kernel(const __grid_constant__ MultiArgs a)
         const TensorEntry &te = a.tensors[t];
         const unsigned long long *row =
             reinterpret_cast<const unsigned long long *>(a.grads) + static_cast<int64_t>(t) * a.W;
-        const int64_t begin = (tile - te.first_tile) * kTile;
         const int64_t size = te.size;
-        if (te.vec == VEC) {
-            const int64_t i = begin + static_cast<int64_t>(threadIdx.x) * VEC;
+        const auto after = snapshots.for_tensor(t);
+        // A vector-aligned tensor with leading elements spends its first tile on
+        // them (through the element path); its later tiles cover the body.
+        const int64_t local = tile - te.first_tile;
+        const int64_t head = te.vec == VEC ? te.head : 0;
+        if (te.vec == VEC && (head == 0 || local > 0)) {
+            const int64_t i = head + (local - (head > 0 ? 1 : 0)) * kTile + static_cast<int64_t>(threadIdx.x) * VEC;
             if (i + VEC <= size) {
                 auto grad_ptr = [&](int slot) -> const void * {
                     return reinterpret_cast<const void *>(__ldg(row + a.sched.member[slot]));
@@ -498,18 +687,34 @@ star_update_multi_kernel(const __grid_constant__ MultiArgs a)
                                  : "l"(which == 0 ? &te.params : &te.momentum));
                     return reinterpret_cast<float *>(base);
                 };
-                update_vector<G, VEC, DEPTH>(state_ptr, i, a.sched, a.hyper, grad_ptr);
+                update_vector<G, VEC, DEPTH, TREE>(state_ptr, i, a.sched, a.hyper, grad_ptr, after);
             } else if (i < size) {                   // the tensor's last, partial vector
-                update_elements<G, DEPTH>(te, row, i, size, 1, a.sched, a.hyper);
+                update_elements<G, DEPTH, TREE>(te, row, i, size, 1, a.sched, a.hyper, after);
             }
         } else {
-            // Not aligned for the full vector width: element by element.  (A
-            // narrower vector path here was measured to cost the aligned path
+            // The leading elements of an aligned tensor, or a tile of a tensor
+            // whose buffers have no common vector alignment: element by element.
+            // (A narrower vector path here was measured to cost the aligned path
             // a third of its bandwidth through register spills.)
-            const int64_t end = min(size, begin + kTile);
-            update_elements<G, DEPTH>(te, row, begin + threadIdx.x, end, kBlockThreads, a.sched, a.hyper);
+            const int64_t begin = te.vec == VEC ? 0 : local * kTile;
+            const int64_t end = te.vec == VEC ? head : min(size, begin + kTile);
+            update_elements<G, DEPTH, TREE>(te, row, begin + threadIdx.x, end, kBlockThreads, a.sched, a.hyper, after);
         }
     }
+}
+
+template <typename G, int VEC, int DEPTH>
+__global__ void __launch_bounds__(kBlockThreads, kResidentBlocks)
+star_update_multi_kernel(const __grid_constant__ MultiArgs a)
+{
+    update_tiles<G, VEC, DEPTH, 0>(a, NoMultiSnapshot());
+}
+
+template <typename G, int VEC, int DEPTH, int TREE>
+__global__ void __launch_bounds__(kBlockThreads, tree_resident_blocks(TREE))
+star_update_multi_ex_kernel(const __grid_constant__ MultiExArgs a)
+{
+    update_tiles<G, VEC, DEPTH, TREE>(a.base, MultiSnapshotSource{&a});
 }
 
 }  // namespace star

@@ -187,3 +187,47 @@ def test_bf16_snapshot_narrowing_on_ties_and_extremes(B):
     O.group_update_f32(x.copy(), np.zeros(n, np.float32), [np.zeros(n, np.float32)], [0, 1], [0], 0.1, 0.9, 0.0,
                        snapshots=[want])
     assert np.array_equal(snap.cpu().view(torch.int16).numpy().view(np.uint16), want)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("snap_dtype", [torch.float32, torch.bfloat16])
+def test_views_at_a_common_element_offset(B, dtype, snap_dtype):
+    """Every buffer a view at the same odd element offset into aligned storage
+    (vector body behind a few leading elements), and one with the snapshot
+    out of phase (element path): same bits as the oracle, guard bands intact."""
+    pad = 32
+    for offset in (1, 3, 7, 8, 9, 13):
+        for n in (2, 9, 4099, 70_001):
+            for snap_extra in (0, 1):
+                g = torch.Generator(device="cuda").manual_seed(offset * 1000 + n)
+
+                def carve(dt, std, shift):
+                    raw = torch.full((n + 2 * pad + shift,), float("nan"), dtype=dt, device="cuda")
+                    view = raw[pad + shift: pad + shift + n]
+                    view.copy_(torch.randn(n, generator=g, device="cuda") * std)
+                    return raw, view
+                (p_raw, p), (v_raw, v) = carve(torch.float32, 0.05, offset), carve(torch.float32, 0.02, offset)
+                grads = [carve(dtype, 0.01, offset)[1] for _ in range(6)]
+                s_raw, snap = carve(snap_dtype, 0.0, offset + snap_extra)
+                off, mem, lrs = [0, 5, 6], [4, 0, 5, 2, 1, 3], [0.1, 0.05]
+                for order, name in ((B.STAR_SUM_LINEAR, "linear"), (B.STAR_SUM_TREE, "tree")):
+                    q, u = p.clone(), v.clone()
+                    p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+                    want = [np.zeros(n, np.uint16 if snap_dtype == torch.bfloat16 else np.float32), None]
+                    O.group_update_f32(p_np, v_np, [grad_to_numpy(x) for x in grads], off, mem,
+                                       np.array(lrs, np.float32), 0.9, 1e-3, snapshots=want, sum_order=name)
+                    B.star_group_update_ex(p, v, grads, off, mem, lrs, 0.9, 1e-3, snapshots=[snap, None],
+                                           sum_order=order)
+                    torch.cuda.synchronize()
+                    what = "offset=%d n=%d extra=%d %s" % (offset, n, snap_extra, name)
+                    assert_matches(p, p_np, "params " + what)
+                    assert_matches(v, v_np, "momentum " + what)
+                    if snap_dtype == torch.bfloat16:
+                        assert np.array_equal(snap.cpu().view(torch.int16).numpy().view(np.uint16), want[0]), what
+                    else:
+                        assert_matches(snap, want[0], "snapshot " + what)
+                    for raw, shift in ((p_raw, offset), (v_raw, offset), (s_raw, offset + snap_extra)):
+                        assert bool(torch.isnan(raw[: pad + shift].float()).all()), what
+                        assert bool(torch.isnan(raw[pad + shift + n:].float()).all()), what
+                    p.copy_(q)
+                    v.copy_(u)

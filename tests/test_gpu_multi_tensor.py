@@ -125,3 +125,53 @@ def test_list_round_with_per_group_rates(B):
     assert_matches(torch.cat(momentum), v_np, "momentum")
     with pytest.raises(ValueError):
         B.star_group_update_multi_lrs(plan, off, mem, [0.1], 0.9, 0.01)
+
+
+def test_aliased_list_entries_are_refused(B):
+    """A buffer that a round writes may not share memory with any other buffer
+    of the list, in whichever tensor: different blocks would update it at once."""
+    W, sizes = 2, [1000, 1000, 64]
+    params, momentum, grads = build(sizes, W, torch.bfloat16, seed=4)
+    ws = torch.empty(B.star_multi_workspace_bytes(sizes, W), dtype=torch.uint8, device="cuda")
+    before = B.star_launch_count()
+    tied = list(params)
+    tied[1] = params[0]                               # a tied weight listed twice
+    crossed = list(momentum)
+    crossed[1] = params[0]                            # one tensor's momentum is another's parameters
+    for bad_p, bad_v in ((tied, momentum), (params, crossed)):
+        with pytest.raises(B.StarError) as e:
+            B.star_multi_prepare(bad_p, bad_v, grads, ws)
+        assert e.value.status == B.STAR_ERR_INVALID_ARG
+    read_only = [[torch.zeros(s, dtype=torch.bfloat16, device="cuda") for s in sizes]] * W
+    B.star_multi_prepare(params, momentum, read_only, ws)          # gradients may alias one another
+    written = [list(g) for g in grads]
+    written[1][2] = params[0].view(torch.bfloat16)[:64]             # a gradient inside another tensor's parameters
+    with pytest.raises(B.StarError) as e:
+        B.star_multi_prepare(params, momentum, written, ws)
+    assert e.value.status == B.STAR_ERR_INVALID_ARG
+    assert B.star_launch_count() == before
+
+
+def test_prepare_refuses_to_run_inside_a_stream_capture(B):
+    """The table is copied from host memory that is released on return; a graph
+    would read it again at every replay.  The call says so and enqueues nothing;
+    the capture is ended and the graph is never replayed."""
+    W, sizes = 2, [300, 5000]
+    params, momentum, grads = build(sizes, W, torch.bfloat16, seed=5)
+    ws = torch.zeros(B.star_multi_workspace_bytes(sizes, W), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    status = None
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        try:
+            B.star_multi_prepare(params, momentum, grads, ws, stream=side)
+        except B.StarError as e:
+            status = e.status
+        graph.capture_end()
+    torch.cuda.synchronize()
+    assert status == B.STAR_ERR_UNSUPPORTED
+    assert not ws.any()                                # nothing was copied
+    del graph

@@ -112,3 +112,86 @@ def test_limits_and_errors(B):
     B.star_group_update_multi_noalloc(params, momentum, grads, [0], [], 0.1, 0.9, 0.0)     # no-op
     torch.cuda.synchronize()
     assert same_bits(params, p0)
+
+
+def test_refused_inside_a_stream_capture(B):
+    """Called while its stream is being captured the entry point returns
+    STAR_ERR_UNSUPPORTED before it touches the shared table or the caller's
+    tensors; the capture is ended and the graph is never replayed.  A normal
+    call afterwards still matches the workspace path."""
+    sizes, W = [4000, 9, 30_000], 3
+    params, momentum, grads = make_list(sizes, W, torch.bfloat16, seed=11)
+    off, mem = [0, 2, 3], [2, 0, 1]
+    B.star_group_update_multi_noalloc(params, momentum, grads, off, mem, 0.1, 0.9, 1e-4)   # set-up outside capture
+    torch.cuda.synchronize()
+    p0 = [x.clone() for x in params]
+    launches = B.star_launch_count()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    status = None
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        try:
+            B.star_group_update_multi_noalloc(params, momentum, grads, off, mem, 0.1, 0.9, 1e-4, stream=side)
+        except B.StarError as e:
+            status = e.status
+        graph.capture_end()
+    torch.cuda.synchronize()
+    del graph
+    assert status == B.STAR_ERR_UNSUPPORTED
+    assert B.star_launch_count() == launches
+    assert same_bits(params, p0)
+    want_p, want_v = reference(B, params, momentum, grads, off, mem, 0.1, 0.9, 1e-4)
+    B.star_group_update_multi_noalloc(params, momentum, grads, off, mem, 0.1, 0.9, 1e-4)
+    torch.cuda.synchronize()
+    assert same_bits(params, want_p) and same_bits(momentum, want_v)
+
+
+def test_error_found_after_the_table_was_rewritten(B):
+    """Scheduling a worker that has no gradient for some tensor is only seen once
+    the table is in place: nothing is launched, the tensors stay as they were,
+    and the next good call is still right."""
+    sizes, W = [700, 4096], 3
+    params, momentum, grads = make_list(sizes, W, torch.float32, seed=12)
+    holes = [list(g) for g in grads]
+    holes[2][1] = None
+    p0 = [x.clone() for x in params]
+    launches = B.star_launch_count()
+    with pytest.raises(B.StarError) as e:
+        B.star_group_update_multi_noalloc(params, momentum, holes, [0, 3], [0, 1, 2], 0.1, 0.9, 0.0)
+    assert e.value.status == B.STAR_ERR_NULL_POINTER
+    torch.cuda.synchronize()
+    assert B.star_launch_count() == launches and same_bits(params, p0)
+    want_p, want_v = reference(B, params, momentum, holes, [0, 2], [1, 0], 0.1, 0.9, 0.0)
+    B.star_group_update_multi_noalloc(params, momentum, holes, [0, 2], [1, 0], 0.1, 0.9, 0.0)
+    B.star_group_update_multi_noalloc([], [], [[] for _ in range(W)], [0, 1], [0], 0.1, 0.9, 0.0)   # empty list
+    torch.cuda.synchronize()
+    assert same_bits(params, want_p) and same_bits(momentum, want_v)
+
+
+def test_a_list_that_fills_the_fixed_array_exactly(B):
+    """The largest list that still fits: its table needs exactly STAR_STATIC_SCRATCH_BYTES."""
+    W = 1
+    n_tensors = 1
+    while B.star_multi_workspace_bytes([8] * (n_tensors + 1), W) <= B.STAR_STATIC_SCRATCH_BYTES:
+        n_tensors += 1
+    # pad the last step with larger tensors until the table size lands on the limit
+    sizes = [8] * n_tensors
+    assert B.star_multi_workspace_bytes(sizes, W) <= B.STAR_STATIC_SCRATCH_BYTES
+    grow = 0
+    while B.star_multi_workspace_bytes(sizes, W) < B.STAR_STATIC_SCRATCH_BYTES and grow < n_tensors:
+        sizes[grow] = 1024 * 64 + 8                      # 64 more tiles' worth of map entries
+        grow += 1
+    assert B.star_multi_workspace_bytes(sizes, W) == B.STAR_STATIC_SCRATCH_BYTES
+    g = torch.Generator(device="cuda").manual_seed(13)
+    flat_p = torch.randn(sum(sizes), generator=g, device="cuda") * 0.05
+    flat_v = torch.zeros(sum(sizes), device="cuda")
+    flat_g = torch.randn(sum(sizes), generator=g, device="cuda") * 0.01
+    params, momentum, grads = list(flat_p.split(sizes)), list(flat_v.split(sizes)), [list(flat_g.split(sizes))]
+    want_p = flat_p.clone()
+    want_v = flat_v.clone()
+    B.star_group_update(want_p, want_v, [flat_g], [0, 1], [0], 0.1, 0.9, 1e-4)
+    B.star_group_update_multi_noalloc(params, momentum, grads, [0, 1], [0], 0.1, 0.9, 1e-4)
+    torch.cuda.synchronize()
+    assert torch.equal(flat_p, want_p) and torch.equal(flat_v, want_v)
