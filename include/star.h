@@ -187,7 +187,7 @@ STAR_API star_status_t star_choose_mode(const double *iter_time, const int32_t *
  *   iter_time[w]   predicted iteration time in the ring; a worker is a straggler
  *                  iff (t - min t) / min t > straggler_threshold (Section II: 0.2)
  *   child_time[w]  predicted iteration time of w when attached to a parent; a
- *                  removed worker counts (q) iff child_time[w] <= t_ring + t_w
+ *                  removed worker counts (q) iff child_time[w] - t_ring <= t_w
  *   t_w_max        largest wait considered (t_w in [0, t_w_max])
  * The x slowest stragglers are removed (x = 0..X, at least one worker stays);
  * only t_w = 0 and the waits at which one more child makes it are candidates;
@@ -202,6 +202,16 @@ STAR_API star_status_t star_choose_all_reduce_mode(const double *iter_time, cons
                                                    double *t_w_out, double *T_out,
                                                    int32_t *removed_out, int32_t *offsets_out,
                                                    int32_t *members_out, int *n_groups_out);
+
+/* Parents of the workers taken out of the ring (Section IV-B: each removed
+ * straggler reports to a non-straggler with high bandwidth; Section IV-D2a
+ * balances the number of children per parent).  Behind a non-blocking switch
+ * every ring member is equally near, so the removed workers (removed[0..x), in
+ * the order star_choose_all_reduce_mode lists them) are dealt round-robin over
+ * the ring members in ascending worker index.  parent_of_out[W] receives the
+ * parent of each removed worker and -1 for ring members.  0 <= x < W. */
+STAR_API star_status_t star_assign_parents(const int32_t *removed, int x, int W,
+                                           int32_t *parent_of_out);
 
 /* Sharding helper (host only).  The path is elementwise, so a job spread over
  * several parameter servers / GPUs (the paper runs one to N PSs per job,

@@ -109,10 +109,14 @@ def choose_mode(iter_time: Sequence[float], labels: Sequence[int], phi: float,
 #
 # Readings where the paper is silent or loose:
 #   * which x stragglers are removed: the x slowest (ties: larger index first).
-#   * "q = removed stragglers with new iteration times no higher than t_w": a
-#     removed worker w has a predicted iteration time as a child, child_time[w];
-#     it counts iff child_time[w] <= t_ring + t_w, i.e. its report is in before
-#     its parent stops waiting.
+#   * q, which the paper describes as the number of removed stragglers whose
+#     new iteration time does not exceed t_w: a removed worker w has a predicted
+#     iteration time as a child, child_time[w]; t_w is a wait that starts when
+#     the ring's slowest member is done, so w counts iff child_time[w] - t_ring
+#     <= t_w, i.e. its report is in before its parent stops waiting.  (Read
+#     literally, child_time[w] <= t_w, a child would have to finish within the
+#     wait alone; time_all_reduce(..., literal=True) evaluates that reading so
+#     that a test can show where the two part.)
 #   * range of t_w: 0 <= t_w <= t_w_max.  Only t_w = 0 and the values at which
 #     one more child makes it, child_time[w] - t_ring, can be optimal.
 #   * ties: fewer removed workers, then the shorter wait.
@@ -130,13 +134,19 @@ def stragglers(iter_time: Sequence[float], threshold: float = 0.2) -> List[int]:
 
 
 def time_all_reduce(iter_time: Sequence[float], child_time: Sequence[float], removed: Sequence[int],
-                    t_w: float, phi: float, M: float) -> Tuple[float, List[int]]:
+                    t_w: float, phi: float, M: float, literal: bool = False) -> Tuple[float, List[int]]:
     """Eq. 3 for a given set of removed workers and wait time.  Returns (T_a,
-    the removed workers whose gradients still arrive in time)."""
+    the removed workers whose gradients still arrive in time).  The test for
+    "in time" has the form in which the candidate waits are built,
+    child_time - t_ring <= t_w (the sum t_ring + t_w can round below
+    child_time for t_w = child_time - t_ring)."""
     N = len(iter_time)
     ring = [w for w in range(N) if w not in removed]
     t_ring = max(iter_time[w] for w in ring)
-    in_time = [w for w in removed if child_time[w] <= t_ring + t_w]
+    if literal:
+        in_time = [w for w in removed if child_time[w] <= t_w]
+    else:
+        in_time = [w for w in removed if child_time[w] - t_ring <= t_w]
     x, q = len(removed), len(in_time)
     return (1.0 + phi / ((N - x + q) * M / N)) * (t_ring + t_w), in_time
 

@@ -105,6 +105,8 @@ def _load() -> ctypes.CDLL:
     lib.star_choose_mode.restype = c_int
     lib.star_choose_all_reduce_mode.argtypes = [c_vp, c_vp, c_int] + [ctypes.c_double] * 4 + [c_vp] * 7
     lib.star_choose_all_reduce_mode.restype = c_int
+    lib.star_assign_parents.argtypes = [c_vp, c_int, c_int, c_vp]
+    lib.star_assign_parents.restype = c_int
     lib.star_shard_range.argtypes = [c_i64, c_int, c_int, c_i64, c_vp, c_vp]
     lib.star_shard_range.restype = c_int
     lib.star_host_workspace_bytes.argtypes = [c_int, c_int, c_i64, c_vp]
@@ -258,6 +260,13 @@ def star_choose_all_reduce_mode(iter_time: Sequence[float], child_time: Sequence
                                             ctypes.byref(T), removed, offsets, members, ctypes.byref(K)),
            "star_choose_all_reduce_mode")
     return x.value, t_w.value, T.value, list(removed[: x.value]), _unpack(offsets, members, K)
+
+
+def star_assign_parents(removed: Sequence[int], W: int) -> List[int]:
+    """Parent of every worker (-1 for ring members) when ``removed`` leave the ring."""
+    out = _i32([0] * W)
+    _check(_lib.star_assign_parents(_i32(removed), len(removed), W, out), "star_assign_parents")
+    return list(out[:W])
 
 
 def star_shard_range(n: int, world: int, rank: int, align: int = 16) -> Tuple[int, int]:

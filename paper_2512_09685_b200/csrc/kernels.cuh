@@ -618,11 +618,13 @@ struct NoMultiSnapshot {
 
 struct StoreMultiSnapshot {
     const MultiExArgs *a;
-    const unsigned long long *row;     // the tensor's row of the snapshot table
+    int32_t t;                         // the tensor: its row of the snapshot table is looked up at store time
     template <int VEC> __device__ __forceinline__ void operator()(int slot, int64_t first, const float (&p)[VEC]) const
     {
         const int set = a->snapshot_set[slot];
         if (set < 0) return;
+        const unsigned long long *row =
+            reinterpret_cast<const unsigned long long *>(a->snapshots) + static_cast<int64_t>(t) * a->n_sets;
         void *dst = reinterpret_cast<void *>(__ldg(row + set));
         if (dst == nullptr) return;
         if (a->snapshot_bf16) store_bf16<VEC>(static_cast<uint16_t *>(dst) + first, p);
@@ -632,11 +634,7 @@ struct StoreMultiSnapshot {
 
 struct MultiSnapshotSource {
     const MultiExArgs *a;
-    __device__ __forceinline__ StoreMultiSnapshot for_tensor(int32_t t) const
-    {
-        return StoreMultiSnapshot{a, reinterpret_cast<const unsigned long long *>(a->snapshots) +
-                                         static_cast<int64_t>(t) * a->n_sets};
-    }
+    __device__ __forceinline__ StoreMultiSnapshot for_tensor(int32_t t) const { return StoreMultiSnapshot{a, t}; }
 };
 
 // Element-by-element path for the ragged ends of a tensor and for tensors whose

@@ -186,7 +186,7 @@ extern "C" star_status_t star_choose_all_reduce_mode(const double *iter_time, co
         for (double t_w : waits) {
             int q = 0;
             for (int j = 0; j < x; ++j)
-                if (child_time[slow[j]] <= t_ring + t_w) ++q;
+                if (child_time[slow[j]] - t_ring <= t_w) ++q;      // the form the candidate waits are built in
             const double T = (1.0 + phi / (static_cast<double>(W - x + q) * M / N)) * (t_ring + t_w);
             if (!have || T < best_T) {          // strict: ties keep fewer removals, then the shorter wait
                 have = true;
@@ -210,9 +210,30 @@ extern "C" star_status_t star_choose_all_reduce_mode(const double *iter_time, co
     // One group: the ring members and the children whose reports are in on time.
     int32_t count = 0;
     for (int w = 0; w < W; ++w)
-        if (!is_removed[w] || child_time[w] <= t_ring + best_wait) members_out[count++] = w;
+        if (!is_removed[w] || child_time[w] - t_ring <= best_wait) members_out[count++] = w;
     offsets_out[0] = 0;
     offsets_out[1] = count;
     *n_groups_out = 1;
     return STAR_OK;
 }
+
+// Parents of the removed workers: the j-th removed worker (as listed, slowest
+// first) goes to ring member j mod R of the ring in ascending worker index.
+extern "C" star_status_t star_assign_parents(const int32_t *removed, int x, int W, int32_t *parent_of_out)
+{
+    if (!parent_of_out || (x > 0 && !removed)) return STAR_ERR_NULL_POINTER;
+    if (W < 1 || x < 0 || x >= W) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    std::vector<bool> is_removed(W, false);
+    for (int j = 0; j < x; ++j) {
+        if (removed[j] < 0 || removed[j] >= W || is_removed[removed[j]]) return STAR_ERR_INVALID_ARG;
+        is_removed[removed[j]] = true;
+    }
+    std::vector<int32_t> ring;
+    for (int w = 0; w < W; ++w)
+        if (!is_removed[w]) ring.push_back(w);
+    for (int w = 0; w < W; ++w) parent_of_out[w] = -1;
+    for (int j = 0; j < x; ++j) parent_of_out[removed[j]] = ring[static_cast<size_t>(j) % ring.size()];
+    return STAR_OK;
+}
+

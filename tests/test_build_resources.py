@@ -41,3 +41,24 @@ def test_hot_kernels_fit_four_blocks_per_sm_without_spills():
     for name in hot:
         assert report[name]["regs"] <= 64, (name, report[name])
         assert report[name]["spill"] == 0, (name, report[name])
+
+
+def test_extended_and_reduce_kernels_do_not_spill():
+    """The snapshot / tree-order kernels of the flat entry point and the group
+    reduce kernels, every instantiation: no spills; the variants for groups of up
+    to 4 members keep the 64-register budget of the linear kernels, the larger
+    tree variants are compiled for two blocks per SM (<= 128 registers).  The
+    tensor-list variants may save a few registers around their out-of-line
+    element path, nothing more."""
+    report = ptxas_report()
+    flat = {n: r for n, r in report.items()
+            if "star_update_flat_snapshot_kernel" in n or "star_group_reduce_kernel" in n}
+    assert len(flat) == 2 * 2 * 4 + 2 * 2 * 4, sorted(flat)      # dtype x (vector, element) x tree span, two kernels
+    for name, r in flat.items():
+        tree = int(re.search(r"ELi(\d+)EEEv", name).group(1))
+        assert r["spill"] == 0, (name, r)
+        assert r["regs"] <= (64 if tree <= 4 else 128), (name, r)
+    lists = {n: r for n, r in report.items() if "star_update_multi_ex_kernel" in n}
+    assert len(lists) == 8, sorted(lists)
+    for name, r in lists.items():
+        assert r["spill"] <= 128, (name, r)

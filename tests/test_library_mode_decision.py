@@ -107,3 +107,30 @@ def test_all_reduce_worked_example_through_the_library():
         B.star_choose_all_reduce_mode([1.0, 2.0], [1.0], 1.0, 64.0, 0.1)
     with pytest.raises(B.StarError):
         B.star_choose_all_reduce_mode([1.0, 2.0], [1.0, -2.0], 1.0, 64.0, 0.1)
+
+
+def test_rounding_sensitive_wait_through_the_library():
+    t_ring, child = 2.8929907811485323, 7.687996268929637
+    t, c = [t_ring, t_ring] + [100.0] * 8, [1.0, 1.0] + [child] * 8
+    x, t_w, T, removed, (off, mem) = B.star_choose_all_reduce_mode(t, c, 1e9, 64.0, 10.0)
+    wx, wt, wT, wremoved, wused = D.choose_all_reduce_mode(t, c, 1e9, 64.0, 10.0)
+    assert (x, removed, mem) == (8, wremoved, list(range(10))) == (wx, wremoved, wused)
+    assert t_w == wt == child - t_ring and T == pytest.approx(wT, rel=1e-15)
+
+
+def test_parent_assignment_matches_the_round_oracle():
+    from oracle import all_reduce as AR
+    rng = random.Random(8)
+    for _ in range(200):
+        W = rng.randint(1, 16)
+        x = rng.randint(0, W - 1)
+        removed = rng.sample(range(W), x)
+        ring = [w for w in range(W) if w not in removed]
+        want = AR.assign_parents(removed, ring)
+        got = B.star_assign_parents(removed, W)
+        assert got == [want.get(w, -1) for w in range(W)]
+        counts = [got.count(r) for r in ring]
+        assert max(counts) - min(counts) <= 1                      # children per parent balanced (Section IV-D2a)
+    for removed, W in (([0, 0], 3), ([3], 3), ([0, 1, 2], 3)):
+        with pytest.raises(B.StarError):
+            B.star_assign_parents(removed, W)

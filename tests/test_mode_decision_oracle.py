@@ -129,3 +129,41 @@ def test_breakpoint_enumeration_equals_a_dense_scan_of_wait_times():
         assert T <= dense * (1 + 1e-12)
         assert T == pytest.approx(D.time_all_reduce(t, child, removed, t_w, phi, M)[0])
         assert sorted(set(range(N)) - set(removed)) == [w for w in used if w not in removed]
+
+
+def test_a_child_admitted_by_its_own_wait_exact_rational():
+    """Eq. 3 over the rationals on an input where the float sum t_ring + t_w
+    falls below the child's time for t_w = child_time - t_ring: the wait that is
+    created for a child must admit that child (q = 1), as it does in exact
+    arithmetic, and T_a must be the value Eq. 3 gives for N - x + q = N."""
+    from fractions import Fraction
+    t_ring, child = 2.8929907811485323, 7.687996268929637
+    assert t_ring + (child - t_ring) < child                       # the rounding that used to drop the child
+    # (by Sterbenz's lemma that needs child > 2 t_ring; waiting that long pays when many reports ride on it)
+    N, x_want = 10, 8
+    t = [t_ring, t_ring] + [100.0] * x_want                        # workers 2..9 are the stragglers
+    child_time = [1.0, 1.0] + [child] * x_want
+    phi, M = 1e9, 64.0                                             # noisy gradients: the eight reports are worth the wait
+    x, t_w, T, removed, used = D.choose_all_reduce_mode(t, child_time, phi, M, t_w_max=10.0)
+    assert (x, sorted(removed), used) == (x_want, list(range(2, N)), list(range(N)))
+    assert t_w == child - t_ring
+    F = Fraction
+    exact = (1 + F(phi) / (F(N - x_want + x_want) * F(M) / N)) * (F(t_ring) + F(t_w))
+    assert T == pytest.approx(float(exact), rel=1e-15)
+    dropped = (1 + F(phi) / (F(N - x_want) * F(M) / N)) * (F(t_ring) + F(t_w))
+    assert float(dropped) > T * 4                                  # what undercounting q would have reported
+
+
+def test_where_the_literal_reading_of_q_parts_from_the_one_taken():
+    """Read literally, a removed worker counts only if its whole iteration as a
+    child fits into the wait t_w; the reading taken counts it if it is done t_w
+    after the ring.  A child that needs 1.2 when the ring needs 1.0: a wait of
+    0.2 admits it under the reading taken, not under the literal one (which
+    would need a wait of 1.2, longer than a ring iteration)."""
+    t, child, phi, M = [1.0, 1.0, 4.0], [9.0, 9.0, 1.2], 1e4, 128.0
+    T_taken, in_taken = D.time_all_reduce(t, child, [2], 0.2, phi, M)
+    T_literal, in_literal = D.time_all_reduce(t, child, [2], 0.2, phi, M, literal=True)
+    assert in_taken == [2] and in_literal == []
+    assert T_taken == pytest.approx((1 + phi / (3 * M / 3)) * 1.2)
+    assert T_literal == pytest.approx((1 + phi / (2 * M / 3)) * 1.2)
+    assert D.time_all_reduce(t, child, [2], 1.2, phi, M, literal=True)[1] == [2]
