@@ -17,7 +17,12 @@ def test_reference_arm_prints_one_json_line_with_the_contract_keys():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["unit"] == "GB/s" and d["higher_is_better"] is True
     assert d["steps"] == 3 and d["warmup"] == 1 and d["value"] > 0 and d["ms_per_step"] > 0
-    assert d["config"]["workload"] == "cfg1_resnet50" and d["vs_baseline"] is None
+    assert d["config"]["workload"] == "cfg4_gpt2_medium" and d["vs_baseline"] is None
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2512_09685_b200 import workloads as WL
+    assert d["config"] == bench.config_for(WL.BY_NAME["cfg4_gpt2_medium"], 1)     # what the GPU arm prints too
+    assert d["config"]["bytes_per_step"] == 354_823_168 * (16 * 2 + 16)
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
     assert d["cpu_baseline"]["value"] == d["value"]
     assert d["e2e"] == {"value": d["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}

@@ -100,3 +100,19 @@ def test_bench_line_on_a_small_case():
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert r["traffic"] is None                        # reduced size: no capture applies
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    regions = d["timed_regions"]
+    assert regions["count"] >= 3 and regions["steps_each"] == 5
+    assert regions["value_min"] <= d["value"] <= regions["value_max"]
+    assert d["config"]["workload"] == "cfg4_gpt2_medium" and d["roofline"]["kernel"] == "star_update_multi_kernel"
+
+
+def test_all_reduce_architecture_round_on_one_gpu():
+    """One rank: a ring of one, nobody removed -- the aggregate and update
+    kernels of the round still run (two launches per step)."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--architecture", "all_reduce",
+                          "--steps", "5", "--warmup", "3", "--n", "4000000"], capture_output=True, text=True,
+                         timeout=600, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    d = json.loads([l for l in out.stdout.splitlines() if l.strip()][-1])
+    assert d["config"]["architecture"] == "all_reduce" and d["n_gpus"] == 1
+    assert d["gpu_launches"] == 10 and d["value"] > 100
