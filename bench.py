@@ -599,16 +599,23 @@ def extra_entry(t, steps: int, peak: float, peak_kind: str, kernel: str, n: int,
     return out
 
 
-def time_other_workloads(headline, peak: float, peak_kind: str):
+def time_other_workloads(headline, peak: float, peak_kind: str, only=None, n_synthetic: int = 100_000_000):
     """The remaining bar workloads, the extended entry points and the kernels of
-    the all-reduce round, each timed like the headline (rank 0, one GPU)."""
+    the all-reduce round, each timed like the headline (rank 0, one GPU).
+    `only`: run just the entry of that name; `n_synthetic`: elements of the
+    entries that are not one of the five workloads (smaller for profiler captures)."""
     import dataclasses
     import torch
     from paper_2512_09685_b200 import binding as B
     from paper_2512_09685_b200 import workloads as WL
     others = {}
 
+    def wanted(name):
+        return only is None or only == name
+
     def run(name, w, mode="plain", note=""):
+        if not wanted(name):
+            return None
         big = w.n > 30_000_000
         dw = DeviceWorkload(w, grad_sets=1 if big else 8, mode=mode)
         steps = 50 if big else 400
@@ -620,7 +627,7 @@ def time_other_workloads(headline, peak: float, peak_kind: str):
         if other.name == headline.name:
             continue
         dw = run(other.name, other)
-        if other.n <= 30_000_000 and not other.multi_tensor and other.n * (other.W * other.grad_bytes + 16) < 126e6:
+        if dw is not None and other.n <= 30_000_000 and not other.multi_tensor and other.n * (other.W * other.grad_bytes + 16) < 126e6:
             # L2-resident, launch-bound size: also the same rounds replayed from a
             # CUDA graph (schedules encoded once at capture), i.e. without the host.
             others[other.name]["note"] = "working set fits L2: not an HBM figure"
@@ -639,7 +646,7 @@ def time_other_workloads(headline, peak: float, peak_kind: str):
         del del_me
         torch.cuda.empty_cache()
     # Tree order on one group of 16 (the 8-leaf-block kernel, two blocks per SM), 100 M elements.
-    one16 = dataclasses.replace(WL.scaled(WL.BY_NAME["cfg2_bert_large"], 100_000_000), name="tree_1x16_100M",
+    one16 = dataclasses.replace(WL.scaled(WL.BY_NAME["cfg2_bert_large"], n_synthetic), name="tree_1x16_100M",
                                 schedule="fixed", fixed_labels=(0,) * 16)
     del_me = run("tree_1x16_100M", one16, "tree", "one group of 16 workers in tree order")
     del del_me
@@ -652,10 +659,14 @@ def time_other_workloads(headline, peak: float, peak_kind: str):
         torch.cuda.empty_cache()
 
     # The two kernels of the all-reduce round, 100 M elements of bf16 gradients.
-    n = 100_000_000
+    n = n_synthetic
+    if only is not None and not (only.startswith("group_reduce") or only.startswith("update_from_sums")):
+        return others
     grads = [(torch.randn(n, device="cuda") * 0.01).to(torch.bfloat16) for _ in range(4)]
     out = torch.empty(n, device="cuda")
     for count in (2, 4):
+        if not wanted("group_reduce_%d_bf16_to_f32_100M" % count):
+            continue
         nbytes = n * (count * 2 + 4)
         t = time_steps(lambda: (B.star_group_reduce(out, grads, list(range(count))), nbytes)[1], 50, 5, None,
                        launch_count=B.star_launch_count, probe=False)
@@ -663,6 +674,8 @@ def time_other_workloads(headline, peak: float, peak_kind: str):
             t, 50, peak, peak_kind, "star_group_reduce_kernel", n,
             "a parent's aggregate of its own and %d children's gradients; bytes n*(%d*2+4)" % (count - 1, count))
     del grads
+    if not wanted("update_from_sums_R4_100M"):
+        return others
     sums = [torch.randn(n, device="cuda") * 0.01 for _ in range(4)]
     p, v = torch.randn(n, device="cuda") * 0.05, torch.zeros(n, device="cuda")
     nbytes = n * (4 * 4 + 16)
@@ -737,6 +750,7 @@ def run_all_reduce_architecture(args, rank: int, world: int, local_rank: int):
 
 
 def main():
+    global MIN_TIMED_SECONDS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
@@ -752,6 +766,12 @@ def main():
                     help="run the workload at a reduced size (flat: this many elements; tensor list: 2 "
                          "layers and n/1024 vocabulary rows): small cases for profiler captures, "
                          "not a benchmark configuration")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="device time to accumulate over repeated timed regions (0: three regions; for "
+                         "profiler captures)")
+    ap.add_argument("--only", default=None,
+                    help="time just this entry of other_workloads (with --n: its synthetic entries at that "
+                         "size) and print it; for profiler captures of the other kernels")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-extra", action="store_true",
                     help="device-timed headline only: skip the end-to-end leg, the other workloads "
@@ -765,6 +785,7 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank, world)
         return
+    MIN_TIMED_SECONDS = args.min_seconds
 
     import torch
     from paper_2512_09685_b200 import binding as B        # raises if the CUDA library is missing
@@ -790,6 +811,11 @@ def main():
         # tensor list with 2 layers and a vocabulary of n / 1024 rows
         w = WL.reduced_list(w, 2, max(args.n // 1024, 1)) if w.multi_tensor else WL.scaled(w, args.n)
     peak, peak_kind = measured_peak()
+    if args.only:
+        entry = time_other_workloads(w, peak, peak_kind, args.only,
+                                     args.n if args.n > 0 else 100_000_000)
+        print(json.dumps({"other_workloads": entry}), flush=True)
+        return
     dw = DeviceWorkload(w, grad_sets=2 if w.n * w.W * w.grad_bytes < (4 << 30) else 1)
     sampler = ClockSampler(local_rank)
     t = time_device(dw, args.steps, args.warmup, dist, sampler)

@@ -390,6 +390,11 @@ star_status_t dispatch_reduce(ReduceArgs &args, const VectorPlan &plan, int tree
 {
     args.head = plan.head;
     const bool vec = plan.vec == VEC;
+    if (vec && args.count <= 2) {          // too few loads per vector: two vectors per thread
+        static Geometry cache[kMaxDevices];
+        return launch_grid_stride(star_group_reduce_pair_kernel<G, VEC>, cache, args, (args.n - args.head) / VEC / 2,
+                                  stream);
+    }
     switch (tree) {
     case 4: return vec ? launch_reduce<G, VEC, 4>(args, stream) : launch_reduce<G, 1, 4>(args, stream);
     case 16: return vec ? launch_reduce<G, VEC, 16>(args, stream) : launch_reduce<G, 1, 16>(args, stream);

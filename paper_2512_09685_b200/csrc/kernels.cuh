@@ -574,6 +574,48 @@ star_group_reduce_kernel(const __grid_constant__ ReduceArgs a)
     }
 }
 
+// One or two sources (a parent without children, or with one: the common case
+// when few workers are removed): a thread would have only one or two loads in
+// flight, too few to cover the memory latency at any occupancy, so each thread
+// takes two vectors per pass and issues the loads of both before it adds.
+template <typename G, int VEC>
+__global__ void __launch_bounds__(kBlockThreads, kResidentBlocks)
+star_group_reduce_pair_kernel(const __grid_constant__ ReduceArgs a)
+{
+    constexpr int GB = VEC * G::kBytes;
+    const int64_t n_vec = (a.n - a.head) / VEC;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlockThreads;
+    const bool two_sources = a.count > 1;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kBlockThreads + threadIdx.x; i < n_vec; i += 2 * stride) {
+        const int64_t first[2] = {a.head + i * VEC, a.head + (i + stride) * VEC};
+        const bool second = i + stride < n_vec;
+        Raw<GB> raw[2][2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (u == 0 || second) {
+                raw[u][0] = load_stream<GB>(static_cast<const char *>(a.src[0]) + first[u] * G::kBytes);
+                if (two_sources) raw[u][1] = load_stream<GB>(static_cast<const char *>(a.src[1]) + first[u] * G::kBytes);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (u == 0 || second) {
+                float sum[VEC];
+                G::template widen<VEC>(raw[u][0], sum);
+                if (two_sources) {
+                    float f[VEC];
+                    G::template widen<VEC>(raw[u][1], f);
+                    add_rows<VEC>(sum, f);
+                }
+                if (a.out_bf16) store_bf16<VEC>(static_cast<uint16_t *>(a.out) + first[u], sum);
+                else store_state<VEC>(static_cast<float *>(a.out) + first[u], sum);
+            }
+        }
+    }
+    const int64_t e = edge_element<VEC>(a.n, a.head, n_vec);
+    if (e >= 0) reduce_vector<G, 1, 4, 0>(a, e);
+}
+
 // ---------------------------------------------------------------------------
 // Tensor list.  The device workspace holds, in this order (each array 256-byte
 // aligned): per-tensor TensorEntry records, the gradient pointer table

@@ -67,6 +67,8 @@ def test_reduce_every_tail_length(B, dtype, out_dtype):
         grads = [(torch.randn(n, generator=gen, device="cuda") * 0.01).to(dtype) for _ in range(W)]
         for order in (B.STAR_SUM_LINEAR, B.STAR_SUM_TREE):
             check_reduce(B, grads, [4, 0, 5, 2, 1], out_dtype, order, n, what="n=%d order=%d" % (n, order))
+        check_reduce(B, grads, [3, 5], out_dtype, B.STAR_SUM_LINEAR, n, what="n=%d two members" % n)
+        check_reduce(B, grads, [1], out_dtype, B.STAR_SUM_LINEAR, n, what="n=%d one member" % n)
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
@@ -95,8 +97,9 @@ def test_reduce_at_every_alignment(B, dtype):
                 carved = [carve(n, dtype, offset + spread * w, f) for w, f in enumerate(fills)]
                 grads = [view for _, view in carved]
                 for out_dtype in (torch.float32, torch.bfloat16):
-                    check_reduce(B, grads, [2, 0, 3, 1], out_dtype, B.STAR_SUM_LINEAR, n, out_offset=offset,
-                                 what="n=%d offset=%d spread=%d" % (n, offset, spread))
+                    for members in ([2, 0, 3, 1], [3, 1], [2]):     # [3, 1] and [2]: the two-vectors-per-thread kernel
+                        check_reduce(B, grads, members, out_dtype, B.STAR_SUM_LINEAR, n, out_offset=offset,
+                                     what="n=%d offset=%d spread=%d members=%r" % (n, offset, spread, members))
                 for w, (raw, _) in enumerate(carved):
                     assert guards_intact(raw, n, offset + spread * w)
 
