@@ -59,6 +59,8 @@ MAX_REPEATS = 50
 # capture was taken on: once the sources differ the figure is stale and
 # `traffic` is reported as null.
 NCU_TRAFFIC_PER_ELEMENT = {
+    "cfg4_gpt2_medium": (1646.59e6 / 34_631_680, "c2335229b4fd9c9448c332b3b94d9094a4f502ad2c1aad14dd022d82522de2db"),
+    "cfg1_resnet50": (788.21e6 / 25_557_032, "c2335229b4fd9c9448c332b3b94d9094a4f502ad2c1aad14dd022d82522de2db"),
 }
 
 
