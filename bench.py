@@ -210,6 +210,8 @@ class DeviceWorkload:
                     self.plans.append(B.star_multi_prepare_ex(self.params, self.momentum, one, self.snapshots, ws))
         else:
             self.flat_grads = [[bufs[0] for bufs in one] for one in self.grad_sets]
+            # pointers marshalled once per gradient set: the per-round host work is the schedule
+            self.flat_rounds = [B.FlatRoundBuffers(self.params[0], self.momentum[0], g) for g in self.flat_grads]
         self.step_index = 0
         torch.cuda.synchronize()
 
@@ -226,8 +228,7 @@ class DeviceWorkload:
             if self.plans is not None:
                 B.star_group_update_multi(self.plans[which], off, mem, w.lr, w.mu, w.wd)
             else:
-                B.star_group_update(self.params[0], self.momentum[0], self.flat_grads[which], off, mem,
-                                    w.lr, w.mu, w.wd)
+                self.flat_rounds[which].star_group_update(off, mem, w.lr, w.mu, w.wd)
         elif self.plans is not None:
             B.star_group_update_multi_ex(self.plans[which], off, mem, [w.lr] * K, w.mu, w.wd,
                                          list(range(K)) if n_snap else None, order)

@@ -339,6 +339,29 @@ def star_group_update(params: torch.Tensor, momentum: torch.Tensor,
                                   _stream(stream)), "star_group_update")
 
 
+class FlatRoundBuffers:
+    """The buffers of a flat round marshalled once: for callers that run many
+    rounds on the same tensors (only the schedule and the scalars change per
+    round), which saves building the pointer array and re-checking the tensors
+    on every call -- on launch-bound sizes that is most of the host time.  Holds
+    references to the tensors; computes nothing."""
+
+    def __init__(self, params: torch.Tensor, momentum: torch.Tensor, grads: Sequence[Optional[torch.Tensor]]):
+        self.n = params.numel()
+        self.p, self.v = _state(params, "params"), _state(momentum, "momentum")
+        if momentum.numel() != self.n:
+            raise ValueError("params and momentum differ in size")
+        self.W = len(grads)
+        self.ptrs, self.dtype = _grad_pointers(grads, self.n)
+        self._keep = (params, momentum, list(grads))
+
+    def star_group_update(self, group_offsets: Sequence[int], group_members: Sequence[int], lr: float, mu: float,
+                          wd: float, stream=None) -> None:
+        K = len(group_offsets) - 1 if len(group_offsets) else 0
+        _check(_lib.star_group_update(self.p, self.v, self.ptrs, self.W, self.dtype, self.n, _i32(group_offsets),
+                                      _i32(group_members), K, lr, mu, wd, _stream(stream)), "star_group_update")
+
+
 def star_group_update_ex(params: torch.Tensor, momentum: torch.Tensor,
                          grads: Sequence[Optional[torch.Tensor]], group_offsets: Sequence[int],
                          group_members: Sequence[int], lrs: Sequence[float], mu: float, wd: float,

@@ -210,3 +210,35 @@ def test_whole_round_equals_the_round_oracle(B, dtype):
     assert reports == len(ring) + len(in_time) == 8
     assert_matches(p, p_np, "params")
     assert_matches(v, v_np, "momentum")
+
+
+def test_round_at_the_resnet50_size_every_element(B):
+    """An all-reduce round on the ResNet-50-sized workload (8 workers, bf16): two
+    workers removed, one in time; every element of the aggregates, p and v."""
+    from paper_2512_09685_b200 import workloads as WL
+    w = WL.BY_NAME["cfg1_resnet50"]
+    n = w.n
+    p = WL.make_params(w, "cuda")[0]
+    v = WL.make_momentum(w, "cuda")[0]
+    grads = [g[0] for g in WL.make_grads(w, 0, "cuda")]
+    x, t_w, T, removed, (off, mem) = B.star_choose_all_reduce_mode(
+        [1.0, 1.02, 3.0, 0.98, 1.0, 1.05, 5.0, 1.01], [9.0] * 2 + [2.5] + [9.0] * 3 + [1.1, 9.0], 1e4, 256.0, 0.5)
+    assert removed == [6, 2] and mem == [0, 1, 3, 4, 5, 6, 7]        # worker 2 misses the wait
+    parent_of = B.star_assign_parents(removed, w.W)
+    ring = [r for r in range(w.W) if parent_of[r] < 0]
+    in_time = [c for c in removed if c in mem]
+    p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+    want_aggr, reports = AR.all_reduce_round_f32(p_np, v_np, [grad_to_numpy(g) for g in grads], ring,
+                                                 AR.assign_parents(removed, ring), in_time, w.lr, w.mu, w.wd)
+    aggregates = []
+    for r in ring:
+        a = torch.empty(n, device="cuda")
+        B.star_group_reduce(a, grads, [r] + sorted(c for c in in_time if parent_of[c] == r))
+        aggregates.append(a)
+    B.star_group_update_from_sums(p, v, aggregates, reports, w.lr, w.mu, w.wd)
+    torch.cuda.synchronize()
+    assert reports == 7
+    for a, want in zip(aggregates, want_aggr):
+        assert_matches(a, want, "aggregate")
+    assert_matches(p, p_np, "params")
+    assert_matches(v, v_np, "momentum")

@@ -109,3 +109,76 @@ def test_cfg4_gpt2_medium_tensor_list_sampled(B):
     assert all(bool(torch.isfinite(p).all()) for p in params)
     assert all(bool((v != 0).float().mean() > 0.99) for v in momentum)
     assert len(ks) >= 2
+
+
+@pytest.mark.parametrize("mode", ["snap_f32", "snap_bf16", "tree"])
+def test_cfg1_extended_entry_point_every_element(B, mode):
+    """The ResNet-50-sized workload through star_group_update_ex as the benchmark
+    times it (one snapshot per group, or tree order): every element of p, v and
+    of every snapshot, two rounds."""
+    w = WL.BY_NAME["cfg1_resnet50"]
+    n = w.n
+    p = WL.make_params(w, "cuda")[0]
+    v = WL.make_momentum(w, "cuda")[0]
+    p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+    grads = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(w.W)]
+    snap_dtype = {"snap_f32": torch.float32, "snap_bf16": torch.bfloat16}.get(mode)
+    for step in range(2):
+        for wk in range(w.W):
+            WL.fill_grads(w, step, wk, [grads[wk]])
+        off, mem = B.encode(w.decision(step))
+        K = len(off) - 1
+        lrs = [w.lr * (k + 1) / K for k in range(K)]              # distinct rates per group
+        snaps = [torch.empty(n, dtype=snap_dtype, device="cuda") for _ in range(K)] if snap_dtype else None
+        B.star_group_update_ex(p, v, grads, off, mem, lrs, w.mu, w.wd, snapshots=snaps,
+                               sum_order=B.STAR_SUM_TREE if mode == "tree" else B.STAR_SUM_LINEAR)
+        want = None
+        if snap_dtype:
+            want = [np.zeros(n, np.uint16 if snap_dtype == torch.bfloat16 else np.float32) for _ in range(K)]
+        O.group_update_f32(p_np, v_np, [grad_to_numpy(g) for g in grads], off, mem, np.array(lrs, np.float32),
+                           w.mu, w.wd, snapshots=want, sum_order="tree" if mode == "tree" else "linear")
+        torch.cuda.synchronize()
+        assert_matches(p, p_np, "%s step %d params" % (mode, step))
+        assert_matches(v, v_np, "%s step %d momentum" % (mode, step))
+        for k in range(K if snap_dtype else 0):
+            if snap_dtype == torch.bfloat16:
+                got = snaps[k].cpu().view(torch.int16).numpy().view(np.uint16)
+                assert np.array_equal(got, want[k]), "%s step %d snapshot %d" % (mode, step, k)
+            else:
+                assert_matches(snaps[k], want[k], "%s step %d snapshot %d" % (mode, step, k))
+
+
+def test_cfg4_list_with_snapshot_sets_sampled(B):
+    """The GPT-2-medium list through star_group_update_multi_ex as the benchmark
+    times it (per-group rates, one bf16 snapshot set per group): sampled elements
+    of p, v and of every written snapshot set, two rounds."""
+    w = WL.BY_NAME["cfg4_gpt2_medium"]
+    sizes, dev = w.sizes, "cuda"
+    params = WL.make_params(w, dev)
+    momentum = WL.make_momentum(w, dev)
+    grads = [[torch.empty(s, dtype=torch.bfloat16, device=dev) for s in sizes] for _ in range(w.W)]
+    sets = [[torch.zeros(s, dtype=torch.bfloat16, device=dev) for s in sizes] for _ in range(8)]
+    ws = torch.empty(B.star_multi_workspace_bytes_ex(sizes, w.W, 8), dtype=torch.uint8, device=dev)
+    plan = B.star_multi_prepare_ex(params, momentum, grads, sets, ws)
+    idx = [torch.from_numpy(sample_indices(s, 2000 + t, chunk=2048, n_chunks=4)).to(dev) for t, s in enumerate(sizes)]
+    gather = lambda tensors: torch.cat([x[i] for x, i in zip(tensors, idx)])
+    p_ref, v_ref = gather(params).cpu().numpy().copy(), gather(momentum).cpu().numpy().copy()
+    for step in range(2):
+        for wk in range(w.W):
+            WL.fill_grads(w, step, wk, grads[wk])
+        off, mem = B.encode(w.decision(step))
+        K = len(off) - 1
+        lrs = [w.lr * (1 + k) for k in range(K)]
+        choice = [(k * 3) % 8 for k in range(K)]                  # distinct sets, not in order
+        before = B.star_launch_count()
+        B.star_group_update_multi_ex(plan, off, mem, lrs, w.mu, w.wd, choice, B.STAR_SUM_LINEAR)
+        assert B.star_launch_count() == before + 1
+        want = [np.zeros(p_ref.size, np.uint16) for _ in range(K)]
+        O.group_update_f32(p_ref, v_ref, [grad_to_numpy(gather(grads[wk])) for wk in range(w.W)], off, mem,
+                           np.array(lrs, np.float32), w.mu, w.wd, snapshots=want)
+        torch.cuda.synchronize()
+        assert_matches(gather(params), p_ref, "step %d params" % step)
+        assert_matches(gather(momentum), v_ref, "step %d momentum" % step)
+        for k in range(K):
+            got = gather(sets[choice[k]]).cpu().view(torch.int16).numpy().view(np.uint16)
+            assert np.array_equal(got, want[k]), "step %d snapshot of group %d" % (step, k)

@@ -335,3 +335,17 @@ def test_sparse_gradients_with_exact_and_signed_zeros(B, dtype):
         assert_matches(u, want_v, "v wd=%g" % wd)
         assert np.array_equal(np.signbit(u.cpu().numpy()), np.signbit(want_v))
         assert np.array_equal(np.signbit(q.cpu().numpy()), np.signbit(want_p))
+
+
+def test_buffers_marshalled_once_give_the_same_rounds(B):
+    """FlatRoundBuffers forwards to the same entry point with the same pointers."""
+    n = 70_001
+    (_, p), (_, v), grads = make_case(n, 5, torch.bfloat16, seed=31)
+    gl = [g for _, g in grads]
+    q, u = p.clone(), v.clone()
+    rounds = B.FlatRoundBuffers(q, u, gl)
+    for off, mem in (([0, 2, 5], [4, 1, 0, 2, 3]), ([0, 1, 2], [3, 0]), ([0, 5], [0, 1, 2, 3, 4])):
+        B.star_group_update(p, v, gl, off, mem, 0.1, 0.9, 1e-4)
+        rounds.star_group_update(off, mem, 0.1, 0.9, 1e-4)
+    torch.cuda.synchronize()
+    assert torch.equal(p, q) and torch.equal(v, u)
