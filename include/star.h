@@ -444,6 +444,29 @@ STAR_API star_status_t star_group_update_host(float *h_params, float *h_momentum
                                               float mu, float wd, void *d_workspace,
                                               size_t workspace_bytes, void *cuda_stream);
 
+/* The host-buffer round with one learning rate per group (lrs: host, n_groups
+ * values; Section IV-C1), optional parameter snapshots into HOST buffers
+ * (h_snapshots: NULL, or host array of n_groups host pointers, n elements of
+ * snapshot_dtype each, entries may be NULL: the copy of the parameters after
+ * that group's update that the server sends back to the group's workers,
+ * Section II) and the choice of summation order.  Snapshot chunks are staged in
+ * the workspace and copied back with p and v; star_host_workspace_bytes_ex sizes
+ * the workspace for up to max_snapshots snapshots of snapshot_dtype per round.
+ * Everything else as star_group_update_host. */
+STAR_API star_status_t star_host_workspace_bytes_ex(int max_scheduled, star_dtype_t grad_dtype,
+                                                    int max_snapshots, star_dtype_t snapshot_dtype,
+                                                    int64_t chunk_elements, size_t *bytes_out);
+
+STAR_API star_status_t star_group_update_host_ex(float *h_params, float *h_momentum,
+                                                 const void *const *h_grads, int W,
+                                                 star_dtype_t grad_dtype, int64_t n,
+                                                 const int32_t *group_offsets,
+                                                 const int32_t *group_members, int n_groups,
+                                                 const float *lrs, float mu, float wd,
+                                                 void *const *h_snapshots, star_dtype_t snapshot_dtype,
+                                                 star_sum_order_t sum_order, void *d_workspace,
+                                                 size_t workspace_bytes, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------
  * Tensor-list round for callers that cannot allocate device memory.
  *

@@ -114,6 +114,11 @@ def _load() -> ctypes.CDLL:
     lib.star_group_update_host.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
                                            c_f, c_f, c_f, c_vp, ctypes.c_size_t, c_vp]
     lib.star_group_update_host.restype = c_int
+    lib.star_host_workspace_bytes_ex.argtypes = [c_int, c_int, c_int, c_int, c_i64, c_vp]
+    lib.star_host_workspace_bytes_ex.restype = c_int
+    lib.star_group_update_host_ex.argtypes = [c_vp, c_vp, c_vp, c_int, c_int, c_i64, c_vp, c_vp, c_int,
+                                              c_vp, c_f, c_f, c_vp, c_int, c_int, c_vp, ctypes.c_size_t, c_vp]
+    lib.star_group_update_host_ex.restype = c_int
     lib.star_group_update_multi_noalloc.argtypes = [c_int, c_vp, c_vp, c_vp, c_vp, c_int, c_int, c_vp, c_vp,
                                                     c_int, c_f, c_f, c_f, c_vp]
     lib.star_group_update_multi_noalloc.restype = c_int
@@ -649,6 +654,69 @@ def star_group_update_host(params: torch.Tensor, momentum: torch.Tensor,
                                        STAR_DTYPE_F32 if dt is None else dt, n, _i32(group_offsets),
                                        _i32(group_members), K, lr, mu, wd, workspace.data_ptr(),
                                        workspace.numel(), _stream(stream)), "star_group_update_host")
+
+
+def star_host_workspace_bytes_ex(max_scheduled: int, grad_dtype: torch.dtype, max_snapshots: int,
+                                 snapshot_dtype: torch.dtype, chunk_elements: int) -> int:
+    out = ctypes.c_size_t(0)
+    code = lambda dt: STAR_DTYPE_BF16 if dt == torch.bfloat16 else STAR_DTYPE_F32       # noqa: E731
+    _check(_lib.star_host_workspace_bytes_ex(max_scheduled, code(grad_dtype), max_snapshots, code(snapshot_dtype),
+                                             chunk_elements, ctypes.byref(out)), "star_host_workspace_bytes_ex")
+    return out.value
+
+
+def star_group_update_host_ex(params: torch.Tensor, momentum: torch.Tensor,
+                              grads: Sequence[Optional[torch.Tensor]], group_offsets: Sequence[int],
+                              group_members: Sequence[int], lrs: Sequence[float], mu: float, wd: float,
+                              workspace: torch.Tensor, snapshots: Optional[Sequence[Optional[torch.Tensor]]] = None,
+                              sum_order: int = STAR_SUM_LINEAR, stream=None) -> None:
+    """The host-buffer round with per-group rates, host snapshot tensors
+    (``snapshots[k]``: float32 or bfloat16 host tensor or None) and the summation order."""
+    n = params.numel()
+    for t, what in ((params, "params"), (momentum, "momentum")):
+        if t.dtype != torch.float32 or t.is_cuda or not t.is_contiguous():
+            raise TypeError("%s must be a contiguous float32 host tensor" % what)
+    if momentum.numel() != n:
+        raise ValueError("params and momentum differ in size")
+    W = len(grads)
+    ptrs = (ctypes.c_void_p * max(W, 1))()
+    dt = None
+    for w, g in enumerate(grads):
+        if g is None:
+            continue
+        if g.is_cuda or not g.is_contiguous() or g.numel() != n:
+            raise ValueError("gradient %d must be a contiguous host tensor of %d elements" % (w, n))
+        d = _grad_dtype(g)
+        if dt is not None and d != dt:
+            raise TypeError("gradients differ in dtype")
+        dt = d
+        ptrs[w] = g.data_ptr()
+    K = len(group_offsets) - 1 if len(group_offsets) else 0
+    if len(lrs) != K:
+        raise ValueError("need one learning rate per group")
+    snap_arr, snap_dt = None, STAR_DTYPE_F32
+    if snapshots is not None:
+        if len(snapshots) != K:
+            raise ValueError("snapshots needs one entry (tensor or None) per group")
+        snap_arr = (ctypes.c_void_p * max(K, 1))()
+        kinds = set()
+        for k, s in enumerate(snapshots):
+            if s is None:
+                continue
+            if s.is_cuda or not s.is_contiguous() or s.numel() != n:
+                raise ValueError("snapshot %d must be a contiguous host tensor of %d elements" % (k, n))
+            kinds.add(_grad_dtype(s))
+            snap_arr[k] = s.data_ptr()
+        if len(kinds) > 1:
+            raise TypeError("snapshots differ in dtype")
+        snap_dt = kinds.pop() if kinds else STAR_DTYPE_F32
+    if workspace.dtype != torch.uint8 or not workspace.is_cuda or not workspace.is_contiguous():
+        raise TypeError("workspace must be a contiguous uint8 CUDA tensor")
+    _check(_lib.star_group_update_host_ex(params.data_ptr(), momentum.data_ptr(), ptrs, W,
+                                          STAR_DTYPE_F32 if dt is None else dt, n, _i32(group_offsets),
+                                          _i32(group_members), K, (ctypes.c_float * max(K, 1))(*lrs), mu, wd,
+                                          snap_arr, snap_dt, sum_order, workspace.data_ptr(), workspace.numel(),
+                                          _stream(stream)), "star_group_update_host_ex")
 
 
 STAR_STATIC_SCRATCH_BYTES = 1 << 20

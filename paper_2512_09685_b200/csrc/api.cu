@@ -295,6 +295,23 @@ int largest_group(const int32_t *group_offsets, int n_groups)
     return largest;
 }
 
+// The snapshot / tree-order kernel for a tree span (0: linear order).
+star_status_t dispatch_extended(SnapshotArgs &sargs, star_dtype_t grad_dtype, const VectorPlan &plan, int tree,
+                                cudaStream_t stream)
+{
+    const bool bf16 = grad_dtype == STAR_DTYPE_BF16;
+    switch (tree) {
+    case 4: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 4>(sargs, plan, stream)
+                        : dispatch_snapshot<GradF32, kVecF32, 4>(sargs, plan, stream);
+    case 16: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 16>(sargs, plan, stream)
+                         : dispatch_snapshot<GradF32, kVecF32, 16>(sargs, plan, stream);
+    case 64: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 64>(sargs, plan, stream)
+                         : dispatch_snapshot<GradF32, kVecF32, 64>(sargs, plan, stream);
+    default: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 0>(sargs, plan, stream)
+                         : dispatch_snapshot<GradF32, kVecF32, 0>(sargs, plan, stream);
+    }
+}
+
 }  // namespace
 
 extern "C" star_status_t star_group_update(float *params, float *momentum, const void *const *grads, int W,
@@ -356,18 +373,7 @@ extern "C" star_status_t star_group_update_ex(float *params, float *momentum, co
     const int tree = tree_span(sum_order, largest_group(group_offsets, n_groups));
     if (tree == 0 && !any_snapshot)        // per-group rates only
         return dispatch_flat(args, grad_dtype, plan_vector(grad_dtype, buffers, n, true), stream);
-    const VectorPlan plan = plan_vector(grad_dtype, buffers, n, false);
-    const bool bf16 = grad_dtype == STAR_DTYPE_BF16;
-    switch (tree) {
-    case 4: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 4>(sargs, plan, stream)
-                        : dispatch_snapshot<GradF32, kVecF32, 4>(sargs, plan, stream);
-    case 16: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 16>(sargs, plan, stream)
-                         : dispatch_snapshot<GradF32, kVecF32, 16>(sargs, plan, stream);
-    case 64: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 64>(sargs, plan, stream)
-                         : dispatch_snapshot<GradF32, kVecF32, 64>(sargs, plan, stream);
-    default: return bf16 ? dispatch_snapshot<GradBF16, kVecBF16, 0>(sargs, plan, stream)
-                         : dispatch_snapshot<GradF32, kVecF32, 0>(sargs, plan, stream);
-    }
+    return dispatch_extended(sargs, grad_dtype, plan_vector(grad_dtype, buffers, n, false), tree, stream);
 }
 
 // ---------------------------------------------------------------------------
@@ -857,50 +863,41 @@ cudaError_t host_pipeline(int dev, HostPipeline **out)
     return cudaSuccess;
 }
 
-// Bytes of one staging set (p, v and `scheduled` gradient chunks), each
-// sub-buffer rounded up to the workspace alignment.
-size_t host_set_bytes(int scheduled, size_t gsize, int64_t chunk)
+// Bytes of one staging set (p, v, `scheduled` gradient chunks and `snapshots`
+// snapshot chunks), each sub-buffer rounded up to the workspace alignment.
+size_t host_set_bytes(int scheduled, size_t gsize, int snapshots, size_t ssize, int64_t chunk)
 {
     const size_t state = round_up(static_cast<size_t>(chunk) * 4, kWorkspaceAlign);
     const size_t grad = round_up(static_cast<size_t>(chunk) * gsize, kWorkspaceAlign);
-    return 2 * state + static_cast<size_t>(scheduled) * grad;
+    const size_t snap = round_up(static_cast<size_t>(chunk) * ssize, kWorkspaceAlign);
+    return 2 * state + static_cast<size_t>(scheduled) * grad + static_cast<size_t>(snapshots) * snap;
 }
 
-}  // namespace
-
-extern "C" star_status_t star_host_workspace_bytes(int max_scheduled, star_dtype_t grad_dtype,
-                                                   int64_t chunk_elements, size_t *bytes_out)
-{
-    if (!bytes_out) return STAR_ERR_NULL_POINTER;
-    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
-    if (max_scheduled < 0 || chunk_elements < kHostChunkQuantum || chunk_elements % kHostChunkQuantum != 0)
-        return STAR_ERR_INVALID_ARG;
-    if (max_scheduled > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
-    *bytes_out = 2 * host_set_bytes(max_scheduled, grad_dtype == STAR_DTYPE_BF16 ? 2 : 4, chunk_elements);
-    return STAR_OK;
-}
-
-extern "C" star_status_t star_group_update_host(float *h_params, float *h_momentum,
-                                                const void *const *h_grads, int W,
-                                                star_dtype_t grad_dtype, int64_t n,
-                                                const int32_t *group_offsets,
-                                                const int32_t *group_members, int n_groups, float lr,
-                                                float mu, float wd, void *d_workspace,
-                                                size_t workspace_bytes, void *cuda_stream)
+// The host-buffer round: chunked, double-buffered.  lrs == nullptr: one rate lr.
+star_status_t host_update(float *h_params, float *h_momentum, const void *const *h_grads, int W,
+                          star_dtype_t grad_dtype, int64_t n, const int32_t *group_offsets,
+                          const int32_t *group_members, int n_groups, float lr, const float *lrs, float mu, float wd,
+                          void *const *h_snapshots, star_dtype_t snapshot_dtype, star_sum_order_t sum_order,
+                          void *d_workspace, size_t workspace_bytes, void *cuda_stream)
 {
     if (n < 0 || W < 0) return STAR_ERR_INVALID_ARG;
     if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (snapshot_dtype != STAR_DTYPE_F32 && snapshot_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (sum_order != STAR_SUM_LINEAR && sum_order != STAR_SUM_TREE) return STAR_ERR_INVALID_ARG;
     if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
-    FlatArgs args;
-    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, lr, &args.sched, nullptr);
+    SnapshotArgs sargs;
+    FlatArgs &args = sargs.flat;
+    const star_status_t st = flatten_schedule(group_offsets, group_members, n_groups, W, lr, &args.sched, lrs);
     if (st != STAR_OK) return st;
     if (n == 0 || n_groups == 0) return STAR_OK;
     if (!h_params || !h_momentum || !h_grads || !d_workspace) return STAR_ERR_NULL_POINTER;
     if (!aligned(d_workspace, kWorkspaceAlign)) return STAR_ERR_INVALID_ARG;
 
     const size_t gsize = grad_dtype == STAR_DTYPE_BF16 ? 2 : 4;
+    const size_t ssize = snapshot_dtype == STAR_DTYPE_BF16 ? 2 : 4;
     const int scheduled = args.sched.n_slots;
     const size_t state_bytes = static_cast<size_t>(n) * 4, grad_bytes = static_cast<size_t>(n) * gsize;
+    const size_t snap_bytes = static_cast<size_t>(n) * ssize;
     if (!aligned(h_params, 4) || !aligned(h_momentum, 4)) return STAR_ERR_INVALID_ARG;
     if (overlaps(h_params, state_bytes, h_momentum, state_bytes)) return STAR_ERR_INVALID_ARG;
     for (int j = 0; j < scheduled; ++j) {
@@ -910,10 +907,32 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
         if (overlaps(g, grad_bytes, h_params, state_bytes) || overlaps(g, grad_bytes, h_momentum, state_bytes))
             return STAR_ERR_INVALID_ARG;
     }
+    // Snapshots: closing slot of the group and host destination, in group order.
+    int snap_slot[STAR_MAX_WORKERS];
+    void *snap_host[STAR_MAX_WORKERS];
+    int n_snap = 0;
+    for (int k = 0; h_snapshots && k < n_groups; ++k) {
+        void *snap = h_snapshots[k];
+        if (!snap) continue;
+        if (!aligned(snap, ssize)) return STAR_ERR_INVALID_ARG;
+        if (overlaps(snap, snap_bytes, h_params, state_bytes) || overlaps(snap, snap_bytes, h_momentum, state_bytes))
+            return STAR_ERR_INVALID_ARG;
+        for (int j = 0; j < scheduled; ++j)
+            if (overlaps(snap, snap_bytes, h_grads[args.sched.member[j]], grad_bytes)) return STAR_ERR_INVALID_ARG;
+        for (int l = 0; l < n_snap; ++l)
+            if (overlaps(snap, snap_bytes, snap_host[l], snap_bytes)) return STAR_ERR_INVALID_ARG;
+        snap_slot[n_snap] = group_offsets[k + 1] - 1;
+        snap_host[n_snap] = snap;
+        ++n_snap;
+    }
+    const int tree = tree_span(sum_order, largest_group(group_offsets, n_groups));
+    const bool extended = tree != 0 || n_snap > 0;
+
     // Largest chunk (multiple of the quantum) whose two staging sets fit.
-    int64_t chunk = static_cast<int64_t>(workspace_bytes / (2 * (8 + static_cast<size_t>(scheduled) * gsize)));
+    const size_t per_element = 8 + static_cast<size_t>(scheduled) * gsize + static_cast<size_t>(n_snap) * ssize;
+    int64_t chunk = static_cast<int64_t>(workspace_bytes / (2 * per_element));
     chunk = chunk / kHostChunkQuantum * kHostChunkQuantum;
-    while (chunk >= kHostChunkQuantum && 2 * host_set_bytes(scheduled, gsize, chunk) > workspace_bytes)
+    while (chunk >= kHostChunkQuantum && 2 * host_set_bytes(scheduled, gsize, n_snap, ssize, chunk) > workspace_bytes)
         chunk -= kHostChunkQuantum;
     if (chunk < kHostChunkQuantum) return STAR_ERR_WORKSPACE_TOO_SMALL;
     const int64_t needed = (n + kHostChunkQuantum - 1) / kHostChunkQuantum * kHostChunkQuantum;
@@ -929,11 +948,16 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
     if (e != cudaSuccess) return cuda_failed(e);
 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const size_t set_bytes = host_set_bytes(scheduled, gsize, chunk);
+    const size_t set_bytes = host_set_bytes(scheduled, gsize, n_snap, ssize, chunk);
     const size_t state_stride = round_up(static_cast<size_t>(chunk) * 4, kWorkspaceAlign);
     const size_t grad_stride = round_up(static_cast<size_t>(chunk) * gsize, kWorkspaceAlign);
+    const size_t snap_stride = round_up(static_cast<size_t>(chunk) * ssize, kWorkspaceAlign);
     char *const base = static_cast<char *>(d_workspace);
     args.hyper = Hyper{mu, wd};
+    args.head = 0;
+    sargs.snapshot_bf16 = snapshot_dtype == STAR_DTYPE_BF16 ? 1 : 0;
+    // staging buffers are aligned: full vector width, no leading elements
+    const VectorPlan plan{grad_dtype == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32, 0};
 
     // The staging sets may still be in use by an earlier call's copy-back
     // (another stream): order this call's first writes after it.
@@ -948,6 +972,8 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
         char *set = base + static_cast<size_t>(b) * set_bytes;
         float *d_p = reinterpret_cast<float *>(set);
         float *d_v = reinterpret_cast<float *>(set + state_stride);
+        char *d_grads = set + 2 * state_stride;
+        char *d_snaps = d_grads + static_cast<size_t>(scheduled) * grad_stride;
         if (index >= 2) {                       // set b was last used by chunk index - 2
             e = cudaStreamWaitEvent(stream, hp->copied_back[b], 0);
             if (e != cudaSuccess) return cuda_failed(e);
@@ -959,18 +985,19 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
         std::memset(args.grads, 0, sizeof args.grads);
         for (int j = 0; j < scheduled; ++j) {
             const int w = args.sched.member[j];
-            char *d_g = set + 2 * state_stride + static_cast<size_t>(j) * grad_stride;
+            char *d_g = d_grads + static_cast<size_t>(j) * grad_stride;
             const char *h_g = static_cast<const char *>(h_grads[w]) + static_cast<size_t>(first) * gsize;
             e = cudaMemcpyAsync(d_g, h_g, static_cast<size_t>(count) * gsize, cudaMemcpyHostToDevice, stream);
             if (e != cudaSuccess) return cuda_failed(e);
             args.grads[w] = d_g;
         }
+        std::memset(sargs.snapshots, 0, sizeof sargs.snapshots);
+        for (int l = 0; l < n_snap; ++l) sargs.snapshots[snap_slot[l]] = d_snaps + static_cast<size_t>(l) * snap_stride;
         args.params = d_p;
         args.momentum = d_v;
         args.n = count;
-        // staging buffers are aligned: full vector width, no leading elements
-        const star_status_t ls = dispatch_flat(
-            args, grad_dtype, VectorPlan{grad_dtype == STAR_DTYPE_BF16 ? kVecBF16 : kVecF32, 0}, stream);
+        const star_status_t ls = extended ? dispatch_extended(sargs, grad_dtype, plan, tree, stream)
+                                          : dispatch_flat(args, grad_dtype, plan, stream);
         if (ls != STAR_OK) return ls;
         e = cudaEventRecord(hp->kernel_done[b], stream);
         if (e != cudaSuccess) return cuda_failed(e);
@@ -980,6 +1007,12 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
         if (e != cudaSuccess) return cuda_failed(e);
         e = cudaMemcpyAsync(h_momentum + first, d_v, static_cast<size_t>(count) * 4, cudaMemcpyDeviceToHost, hp->copy_back);
         if (e != cudaSuccess) return cuda_failed(e);
+        for (int l = 0; l < n_snap; ++l) {
+            char *h_s = static_cast<char *>(snap_host[l]) + static_cast<size_t>(first) * ssize;
+            e = cudaMemcpyAsync(h_s, d_snaps + static_cast<size_t>(l) * snap_stride, static_cast<size_t>(count) * ssize,
+                                cudaMemcpyDeviceToHost, hp->copy_back);
+            if (e != cudaSuccess) return cuda_failed(e);
+        }
         e = cudaEventRecord(hp->copied_back[b], hp->copy_back);
         if (e != cudaSuccess) return cuda_failed(e);
     }
@@ -989,6 +1022,58 @@ extern "C" star_status_t star_group_update_host(float *h_params, float *h_moment
         if (e != cudaSuccess) return cuda_failed(e);
     }
     return STAR_OK;
+}
+
+}  // namespace
+
+extern "C" star_status_t star_host_workspace_bytes_ex(int max_scheduled, star_dtype_t grad_dtype,
+                                                      int max_snapshots, star_dtype_t snapshot_dtype,
+                                                      int64_t chunk_elements, size_t *bytes_out)
+{
+    if (!bytes_out) return STAR_ERR_NULL_POINTER;
+    if (grad_dtype != STAR_DTYPE_F32 && grad_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (snapshot_dtype != STAR_DTYPE_F32 && snapshot_dtype != STAR_DTYPE_BF16) return STAR_ERR_INVALID_ARG;
+    if (max_scheduled < 0 || max_snapshots < 0 || chunk_elements < kHostChunkQuantum ||
+        chunk_elements % kHostChunkQuantum != 0)
+        return STAR_ERR_INVALID_ARG;
+    if (max_scheduled > STAR_MAX_WORKERS || max_snapshots > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    *bytes_out = 2 * host_set_bytes(max_scheduled, grad_dtype == STAR_DTYPE_BF16 ? 2 : 4, max_snapshots,
+                                    snapshot_dtype == STAR_DTYPE_BF16 ? 2 : 4, chunk_elements);
+    return STAR_OK;
+}
+
+extern "C" star_status_t star_host_workspace_bytes(int max_scheduled, star_dtype_t grad_dtype,
+                                                   int64_t chunk_elements, size_t *bytes_out)
+{
+    return star_host_workspace_bytes_ex(max_scheduled, grad_dtype, 0, STAR_DTYPE_F32, chunk_elements, bytes_out);
+}
+
+extern "C" star_status_t star_group_update_host(float *h_params, float *h_momentum,
+                                                const void *const *h_grads, int W,
+                                                star_dtype_t grad_dtype, int64_t n,
+                                                const int32_t *group_offsets,
+                                                const int32_t *group_members, int n_groups, float lr,
+                                                float mu, float wd, void *d_workspace,
+                                                size_t workspace_bytes, void *cuda_stream)
+{
+    return host_update(h_params, h_momentum, h_grads, W, grad_dtype, n, group_offsets, group_members, n_groups, lr,
+                       nullptr, mu, wd, nullptr, STAR_DTYPE_F32, STAR_SUM_LINEAR, d_workspace, workspace_bytes,
+                       cuda_stream);
+}
+
+extern "C" star_status_t star_group_update_host_ex(float *h_params, float *h_momentum,
+                                                   const void *const *h_grads, int W,
+                                                   star_dtype_t grad_dtype, int64_t n,
+                                                   const int32_t *group_offsets,
+                                                   const int32_t *group_members, int n_groups,
+                                                   const float *lrs, float mu, float wd,
+                                                   void *const *h_snapshots, star_dtype_t snapshot_dtype,
+                                                   star_sum_order_t sum_order, void *d_workspace,
+                                                   size_t workspace_bytes, void *cuda_stream)
+{
+    if (n_groups > 0 && !lrs) return STAR_ERR_NULL_POINTER;
+    return host_update(h_params, h_momentum, h_grads, W, grad_dtype, n, group_offsets, group_members, n_groups, 0.0f,
+                       lrs, mu, wd, h_snapshots, snapshot_dtype, sum_order, d_workspace, workspace_bytes, cuda_stream);
 }
 
 // ---------------------------------------------------------------------------

@@ -80,3 +80,54 @@ def test_host_errors(B):
         B.star_host_workspace_bytes(2, torch.bfloat16, 1000)
     torch.cuda.synchronize()
     assert torch.equal(p, p0)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("snap_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("order", ["linear", "tree"])
+def test_host_round_with_rates_snapshots_and_order(B, dtype, snap_dtype, order):
+    """Per-group rates, snapshots into host tensors and the tree order through the
+    chunked host path: the oracle's bits, snapshots included."""
+    n, W = 300_007, 7
+    off, mem = [0, 5, 6, 7], [6, 0, 4, 2, 5, 1, 3]            # a group of 5: tree and linear orders differ
+    lrs = [0.1, 0.025, 0.05]
+    for chunk in (2048, 65536):
+        p, v, grads = host_case(n, W, dtype, seed=chunk % 89 + 3, pinned=True)
+        snaps = [torch.zeros(n, dtype=snap_dtype).pin_memory(), None, torch.zeros(n, dtype=snap_dtype).pin_memory()]
+        p_np, v_np = p.numpy().copy(), v.numpy().copy()
+        snap_np = np.uint16 if snap_dtype == torch.bfloat16 else np.float32
+        want = [np.zeros(n, snap_np), None, np.zeros(n, snap_np)]
+        O.group_update_f32(p_np, v_np, [grad_to_numpy(g) for g in grads], off, mem, np.array(lrs, np.float32),
+                           0.9, 1e-3, snapshots=want, sum_order=order)
+        ws = torch.empty(B.star_host_workspace_bytes_ex(W, dtype, 2, snap_dtype, chunk), dtype=torch.uint8,
+                         device="cuda")
+        B.star_group_update_host_ex(p, v, grads, off, mem, lrs, 0.9, 1e-3, ws, snapshots=snaps,
+                                    sum_order=B.STAR_SUM_TREE if order == "tree" else B.STAR_SUM_LINEAR)
+        torch.cuda.current_stream().synchronize()
+        assert_matches(p, p_np, "params chunk=%d" % chunk)
+        assert_matches(v, v_np, "momentum chunk=%d" % chunk)
+        for k in (0, 2):
+            if snap_dtype == torch.bfloat16:
+                assert np.array_equal(snaps[k].view(torch.int16).numpy().view(np.uint16), want[k]), "snapshot %d" % k
+            else:
+                assert_matches(snaps[k], want[k], "snapshot %d" % k)
+
+
+def test_host_ex_errors(B):
+    p, v, grads = host_case(5000, 2, torch.bfloat16, seed=2, pinned=False)
+    p0 = p.clone()
+    ws = torch.empty(B.star_host_workspace_bytes_ex(2, torch.bfloat16, 1, torch.float32, 2048), dtype=torch.uint8,
+                     device="cuda")
+    with pytest.raises(B.StarError) as e:                      # snapshot buffer is the parameter buffer
+        B.star_group_update_host_ex(p, v, grads, [0, 2], [0, 1], [0.1], 0.9, 0.0, ws, snapshots=[p])
+    assert e.value.status == B.STAR_ERR_INVALID_ARG
+    s = torch.zeros(5000)
+    with pytest.raises(B.StarError) as e:                      # two groups into one buffer
+        B.star_group_update_host_ex(p, v, grads, [0, 1, 2], [0, 1], [0.1, 0.1], 0.9, 0.0, ws, snapshots=[s, s])
+    assert e.value.status == B.STAR_ERR_INVALID_ARG
+    with pytest.raises(B.StarError) as e:                      # two snapshots do not fit a workspace sized for one
+        B.star_group_update_host_ex(p, v, grads, [0, 1, 2], [0, 1], [0.1, 0.1], 0.9, 0.0, ws,
+                                    snapshots=[s, torch.zeros(5000)])
+    assert e.value.status == B.STAR_ERR_WORKSPACE_TOO_SMALL
+    torch.cuda.synchronize()
+    assert torch.equal(p, p0)
