@@ -213,6 +213,17 @@ STAR_API star_status_t star_choose_all_reduce_mode(const double *iter_time, cons
 STAR_API star_status_t star_assign_parents(const int32_t *removed, int x, int W,
                                            int32_t *parent_of_out);
 
+/* Communication tree (Section IV-D2b: the workers of a job form a tree under
+ * the parameter server, or under a parent in the all-reduce architecture;
+ * workers with longer communication latency sit in lower layers; every worker
+ * adds its children's gradients to its own and forwards the sum; the tree is
+ * rebuilt before each iteration).  A fanout-ary tree filled layer by layer in
+ * ascending latency (ties: the smaller worker index first): the `fanout`
+ * quickest workers become children of the root, the next `fanout` children of
+ * the quickest worker, and so on.  parent_of_out[W] receives each worker's
+ * parent, -1 for the root's children.  latency finite, fanout >= 1. */
+STAR_API star_status_t star_build_tree(const double *latency, int W, int fanout, int32_t *parent_of_out);
+
 /* Sharding helper (host only).  The path is elementwise, so a job spread over
  * several parameter servers / GPUs (the paper runs one to N PSs per job,
  * Section III set-up) needs no exchange inside it: rank r of world owns the

@@ -107,6 +107,8 @@ def _load() -> ctypes.CDLL:
     lib.star_choose_all_reduce_mode.restype = c_int
     lib.star_assign_parents.argtypes = [c_vp, c_int, c_int, c_vp]
     lib.star_assign_parents.restype = c_int
+    lib.star_build_tree.argtypes = [c_vp, c_int, c_int, c_vp]
+    lib.star_build_tree.restype = c_int
     lib.star_shard_range.argtypes = [c_i64, c_int, c_int, c_i64, c_vp, c_vp]
     lib.star_shard_range.restype = c_int
     lib.star_host_workspace_bytes.argtypes = [c_int, c_int, c_i64, c_vp]
@@ -271,6 +273,14 @@ def star_assign_parents(removed: Sequence[int], W: int) -> List[int]:
     """Parent of every worker (-1 for ring members) when ``removed`` leave the ring."""
     out = _i32([0] * W)
     _check(_lib.star_assign_parents(_i32(removed), len(removed), W, out), "star_assign_parents")
+    return list(out[:W])
+
+
+def star_build_tree(latency: Sequence[float], fanout: int) -> List[int]:
+    """Parent of every worker (-1 = child of the root) in the latency-ordered tree."""
+    W = len(latency)
+    out = _i32([0] * W)
+    _check(_lib.star_build_tree(_f64(latency), W, fanout, out), "star_build_tree")
     return list(out[:W])
 
 

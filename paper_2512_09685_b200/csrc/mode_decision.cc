@@ -237,3 +237,22 @@ extern "C" star_status_t star_assign_parents(const int32_t *removed, int x, int 
     return STAR_OK;
 }
 
+// Communication tree (Section IV-D2b): workers with longer latency sit lower.
+// A fanout-ary tree filled layer by layer in ascending latency (ties: smaller
+// index first): the `fanout` quickest workers are children of the root, the
+// next `fanout` children of the quickest one, and so on.
+extern "C" star_status_t star_build_tree(const double *latency, int W, int fanout, int32_t *parent_of_out)
+{
+    if (!parent_of_out || (W > 0 && !latency)) return STAR_ERR_NULL_POINTER;
+    if (W < 0 || fanout < 1) return STAR_ERR_INVALID_ARG;
+    if (W > STAR_MAX_WORKERS) return STAR_ERR_UNSUPPORTED;
+    for (int w = 0; w < W; ++w)
+        if (!std::isfinite(latency[w])) return STAR_ERR_INVALID_ARG;
+    std::vector<int32_t> order(W);
+    for (int w = 0; w < W; ++w) order[w] = w;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return latency[a] < latency[b]; });
+    for (int i = 0; i < W; ++i)
+        parent_of_out[order[i]] = i < fanout ? -1 : order[(i - fanout) / fanout];
+    return STAR_OK;
+}
+

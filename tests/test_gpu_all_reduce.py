@@ -242,3 +242,43 @@ def test_round_at_the_resnet50_size_every_element(B):
         assert_matches(a, want, "aggregate")
     assert_matches(p, p_np, "params")
     assert_matches(v, v_np, "momentum")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_round_over_a_communication_tree(B, dtype):
+    """Section IV-D2b on one GPU: every worker's partial sum (own gradient widened,
+    then its children's sums, ascending) with star_group_reduce, the root's sum and
+    update with star_group_update_from_sums, against oracle/tree_round.py."""
+    from oracle import tree_round as TR
+    n, W = 70_003, 11
+    gen = torch.Generator(device="cuda").manual_seed(123)
+    p = torch.randn(n, generator=gen, device="cuda") * 0.05
+    v = torch.randn(n, generator=gen, device="cuda") * 0.02
+    grads = [(torch.randn(n, generator=gen, device="cuda") * 0.01).to(dtype) for _ in range(W)]
+    for fanout in (1, 2, 3, W):
+        latency = [float((7 * w) % W) for w in range(W)]
+        parent_of = B.star_build_tree(latency, fanout)
+        assert parent_of == TR.build_tree(latency, fanout)
+        q, u = p.clone(), v.clone()
+        p_np, v_np = p.cpu().numpy().copy(), v.cpu().numpy().copy()
+        want_sums = TR.tree_round_f32(p_np, v_np, [grad_to_numpy(g) for g in grads], parent_of, 0.05, 0.9, 1e-4)
+        sums = {}
+
+        def partial(w):
+            if w not in sums:
+                own = torch.empty(n, device="cuda")
+                B.star_group_reduce(own, [grads[w]], [0])
+                kids = [c for c in range(W) if parent_of[c] == w]
+                if kids:
+                    total = torch.empty(n, device="cuda")
+                    B.star_group_reduce(total, [own] + [partial(c) for c in kids], list(range(len(kids) + 1)))
+                    own = total
+                sums[w] = own
+            return sums[w]
+        top = [partial(w) for w in range(W) if parent_of[w] < 0]
+        B.star_group_update_from_sums(q, u, top, W, 0.05, 0.9, 1e-4)
+        torch.cuda.synchronize()
+        for w in range(W):
+            assert_matches(partial(w), want_sums[w], "fanout %d partial sum of worker %d" % (fanout, w))
+        assert_matches(q, p_np, "fanout %d params" % fanout)
+        assert_matches(u, v_np, "fanout %d momentum" % fanout)

@@ -134,3 +134,16 @@ def test_parent_assignment_matches_the_round_oracle():
     for removed, W in (([0, 0], 3), ([3], 3), ([0, 1, 2], 3)):
         with pytest.raises(B.StarError):
             B.star_assign_parents(removed, W)
+
+
+def test_tree_construction_matches_the_round_oracle():
+    from oracle import tree_round as TR
+    rng = random.Random(9)
+    for _ in range(300):
+        W, fanout = rng.randint(0, 20), rng.randint(1, 5)
+        latency = [float(rng.randint(0, 6)) for _ in range(W)]        # many ties
+        assert B.star_build_tree(latency, fanout) == TR.build_tree(latency, fanout)
+    with pytest.raises(B.StarError):
+        B.star_build_tree([1.0, 2.0], 0)
+    with pytest.raises(B.StarError):
+        B.star_build_tree([1.0, float("nan")], 2)
