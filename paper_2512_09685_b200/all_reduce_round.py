@@ -68,8 +68,8 @@ class RoundPlan:
 
 
 def _bits(t: torch.Tensor) -> torch.Tensor:
-    """bf16 travels as its bit pattern (every transport moves 16-bit integers)."""
-    return t.view(torch.int16) if t.dtype == torch.bfloat16 else t
+    """bf16 travels as raw bytes (a type every transport moves; the bits arrive unchanged)."""
+    return t.view(torch.uint8) if t.dtype == torch.bfloat16 else t
 
 
 class AllReduceRound:
