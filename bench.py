@@ -824,14 +824,14 @@ def main():
     t = time_device(dw, args.steps, args.warmup, dist, sampler)
     gbs_rank = t["bytes"] / t["seconds"] / 1e9
     value = gbs_rank * world
-    config = config_for(w, world)
-    config["gradient_buffer_sets_rotated"] = len(dw.grad_sets)
+    config = config_for(w, world)                      # identical in the reference arm
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t["seconds"] / args.steps * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": config,
+        "gradient_buffer_sets_rotated": len(dw.grad_sets),
         "timed_regions": {"count": t["repeats"], "steps_each": args.steps, "seconds_total": t["timed_seconds"],
                           "value_min": t["gbs_regions"][0] * world, "value_median": value,
                           "value_max": t["gbs_regions"][-1] * world,

@@ -104,6 +104,10 @@ def test_bench_line_on_a_small_case():
     assert regions["count"] >= 3 and regions["steps_each"] == 5
     assert regions["value_min"] <= d["value"] <= regions["value_max"]
     assert d["config"]["workload"] == "cfg4_gpt2_medium" and d["roofline"]["kernel"] == "star_update_multi_kernel"
+    import bench
+    from paper_2512_09685_b200 import workloads as WL
+    reduced = WL.reduced_list(WL.BY_NAME["cfg4_gpt2_medium"], 2, 4000000 // 1024)
+    assert d["config"] == bench.config_for(reduced, 1)            # the dict the reference arm prints for the same workload
 
 
 def test_all_reduce_architecture_round_on_one_gpu():
