@@ -349,3 +349,35 @@ def test_buffers_marshalled_once_give_the_same_rounds(B):
         rounds.star_group_update(off, mem, 0.1, 0.9, 1e-4)
     torch.cuda.synchronize()
     assert torch.equal(p, q) and torch.equal(v, u)
+
+
+@pytest.mark.parametrize("size", [2, 3, 4, 5, 8, 16, 32, 64])
+def test_group_means_on_extreme_sums(B, size):
+    """The mean of a group whose sum is subnormal, on a rounding tie of the
+    quotient, huge, infinite, NaN or a signed zero: power-of-two group sizes take a
+    multiply by 2^-k in the kernel, the others the IEEE division; both must land
+    on the oracle's s / |G| bit for bit (mu = wd = 0, lr = 1: v = mean, p = p0 - mean)."""
+    probes = np.array([0.0, -0.0, 1e-45, -1e-45, 3e-45, 5e-45, 7e-45, 1.1754944e-38, 1.1754942e-38, 2.3509887e-38,
+                       -2.9387359e-38, 1.0, 1.0 + 2.0 ** -23, 3.0, -7.0, 1e-20, 3.4028235e38, -3.4028235e38,
+                       np.inf, -np.inf, np.nan, 8.5e37, 2.0 ** -126 * 1.5, 2.0 ** -127, 2.0 ** -149 * (size + 1)],
+                      np.float32)
+    n = probes.size
+    # the first member carries the probe, the others are zero: the group's sum IS the probe
+    grads = [torch.from_numpy(probes.copy()).cuda()] + [torch.zeros(n, device="cuda") for _ in range(size - 1)]
+    off, mem = [0, size], list(range(size))
+    for sum_order, name in ((B.STAR_SUM_LINEAR, "linear"), (B.STAR_SUM_TREE, "tree")):
+        p, v = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+        p_np, v_np = np.zeros(n, np.float32), np.zeros(n, np.float32)
+        O.group_update_f32(p_np, v_np, [g.cpu().numpy() for g in grads], off, mem, np.float32(1.0), 0.0, 0.0,
+                           sum_order=name)
+        B.star_group_update_ex(p, v, grads, off, mem, [1.0], 0.0, 0.0, sum_order=sum_order)
+        torch.cuda.synchronize()
+        got_v, got_p = v.cpu().numpy(), p.cpu().numpy()
+        nan = np.isnan(v_np)
+        assert np.array_equal(np.isnan(got_v), nan) and np.array_equal(np.isnan(got_p), np.isnan(p_np))
+        assert np.array_equal(got_v[~nan].view(np.uint32), v_np[~nan].view(np.uint32)), (size, name)
+        ok = ~np.isnan(p_np)
+        assert np.array_equal(got_p[ok].view(np.uint32), p_np[ok].view(np.uint32)), (size, name)
+        want = probes.astype(np.float64) / size                    # and the oracle's mean is the rounded quotient
+        finite = np.isfinite(want) & ~nan
+        assert np.array_equal(v_np[finite], want[finite].astype(np.float32))
