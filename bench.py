@@ -59,8 +59,8 @@ MAX_REPEATS = 50
 # capture was taken on: once the sources differ the figure is stale and
 # `traffic` is reported as null.
 NCU_TRAFFIC_PER_ELEMENT = {
-    "cfg4_gpt2_medium": (1646.59e6 / 34_631_680, "c2335229b4fd9c9448c332b3b94d9094a4f502ad2c1aad14dd022d82522de2db"),
-    "cfg1_resnet50": (788.21e6 / 25_557_032, "c2335229b4fd9c9448c332b3b94d9094a4f502ad2c1aad14dd022d82522de2db"),
+    "cfg4_gpt2_medium": (1644.47e6 / 34_631_680, "03e0fa45a87f327661444bc4c1aff616ef7e6deddd70b78ae0dd5d517a48867b"),
+    "cfg1_resnet50": (787.86e6 / 25_557_032, "03e0fa45a87f327661444bc4c1aff616ef7e6deddd70b78ae0dd5d517a48867b"),
 }
 
 
