@@ -120,3 +120,16 @@ def test_all_reduce_architecture_round_on_one_gpu():
     d = json.loads([l for l in out.stdout.splitlines() if l.strip()][-1])
     assert d["config"]["architecture"] == "all_reduce" and d["n_gpus"] == 1
     assert d["gpu_launches"] == 10 and d["value"] > 100
+
+
+def test_single_entry_runs_used_for_profiler_captures():
+    """`--only NAME --n N`: one entry of other_workloads at a reduced size (the
+    commands the profile summaries were captured with)."""
+    for name, kernel in (("group_reduce_2_bf16_to_f32_100M", "star_group_reduce_kernel"),
+                         ("tree_1x16_100M", "star_update_flat_snapshot_kernel"),
+                         ("cfg4_gpt2_medium/snap_bf16", "star_update_multi_ex_kernel")):
+        out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--n", "2000000", "--only", name],
+                             capture_output=True, text=True, timeout=600, cwd=ROOT)
+        assert out.returncode == 0, out.stderr[-2000:]
+        d = json.loads([l for l in out.stdout.splitlines() if l.strip()][-1])["other_workloads"]
+        assert list(d) == [name] and d[name]["roofline"]["kernel"] == kernel and d[name]["gbs"] > 50
